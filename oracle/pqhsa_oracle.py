@@ -1,0 +1,236 @@
+"""Float64 CPU oracle of the PQ-HSA decode-step attention operator.
+
+TEST INFRASTRUCTURE ONLY.  This file is the yardstick the CUDA library is checked
+against; it is deliberately plain and slow, shares no code with the library, and is
+imported only by the tests, the smoke check and the benchmark's CPU-baseline leg.
+The product path never calls it.
+
+Every function restates one passage of the paper (Section 3, Eq. 1-5) in numpy
+float64, in the paper's order and notation, without blocking, fusion or
+re-ordering:
+
+    O1  position partition S / L / R and the budget k = ceil(rho |R|)   (Sec. 3.2, Eq. 3; App. A "Budgets")
+    O2  q = r_q u_q                                                      (Sec. 3.1)
+    O3  coarse_j = u_q . c_j ,  LUT[m][z] = u_q^(m) . p_{m,z}            (Sec. 3.1, text after Eq. 2)
+    O4  approximate logit of every indexed token                         (Eq. 2)
+    O5  T = the k positions of R with the largest approximate logit     (Eq. 3)
+    O6  exact logits on E = S u L u T from the original keys             (Sec. 3.2)
+    O7  common shift m_0, e_i on E, e~_i on B = R \\ T                    (Sec. 3.2)
+    O8  per-list background mass M_j, Z^_B, N^_B with the stored means   (Eq. 4)
+    O9  y^ = (N_E + N^_B) / (Z_E + Z^_B)                                 (Eq. 5)
+
+Readings where the paper is silent (each also listed in the design doc):
+  * top-k ties: stable, the lower position wins;
+  * rho is given in parts per million and k is computed in integers;
+  * u_q = 0 when r_q = 0;
+  * the list mean that multiplies M_j is the stored mean over all members of the
+    list, selected ones included (Sec. 3.2, last paragraph);
+  * an empty list contributes zero (text after Eq. 4).
+
+Pins (tests/test_oracle_pins.py): brute-force loops on tiny inputs, the ADC sum
+against a dense dot product with the reconstructed key, rho = 1 against textbook
+softmax attention, the exact-reconstruction / constant-value-per-list case against
+textbook attention at any budget, a hand-computed closed form, mass conservation,
+shift and permutation invariance, the budgets the paper prints (1,456 and 2,752
+tokens at 131,072), and top-k against a full sort.  No function here is
+"parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------- O1
+def budget_k(n_indexed: int, budget_ppm: int) -> int:
+    """k = ceil(rho * |R|) with rho = budget_ppm / 10^6, in integers (Eq. 3)."""
+    if n_indexed <= 0:
+        return 0
+    k = (n_indexed * budget_ppm + 999_999) // 1_000_000
+    return min(k, n_indexed)
+
+
+def partition(seq_len: int, n_sink: int = 0, n_local: int = 0):
+    """Sink prefix S, local window L (most recent tokens) and indexed region R
+    (Sec. 3.2).  Returned as position arrays; they are disjoint and cover [0, N)."""
+    n_s = min(n_sink, seq_len)
+    l_start = max(n_s, seq_len - n_local)
+    S = np.arange(0, n_s, dtype=np.int64)
+    R = np.arange(n_s, l_start, dtype=np.int64)
+    L = np.arange(l_start, seq_len, dtype=np.int64)
+    return S, L, R
+
+
+def exact_set_tokens(seq_len: int, n_sink: int, n_local: int, budget_ppm: int,
+                     round_to_page: int = 0) -> int:
+    """Number of tokens attended exactly: |S| + |L| + ceil(rho |R|), optionally
+    rounded up to whole pages (App. A, "Budgets")."""
+    S, L, R = partition(seq_len, n_sink, n_local)
+    total = len(S) + len(L) + budget_k(len(R), budget_ppm)
+    if round_to_page:
+        total = round_to_page * ((total + round_to_page - 1) // round_to_page)
+    return total
+
+
+# --------------------------------------------------------------------------- O2, O3
+def split_query(q: np.ndarray):
+    """q = r_q u_q (Sec. 3.1)."""
+    q = np.asarray(q, dtype=np.float64)
+    r_q = float(np.sqrt(np.sum(q * q)))
+    u_q = q / r_q if r_q > 0.0 else np.zeros_like(q)
+    return r_q, u_q
+
+
+def build_lut(u_q: np.ndarray, centroids: np.ndarray, codebooks: np.ndarray):
+    """coarse[j] = u_q . c_j and LUT[m][z] = u_q^(m) . p_{m,z} (Sec. 3.1).
+
+    centroids [n_list, d]; codebooks [M, n_code, dsub]; subspace m covers the
+    contiguous dims [m*dsub, (m+1)*dsub)."""
+    centroids = np.asarray(centroids, dtype=np.float64)
+    codebooks = np.asarray(codebooks, dtype=np.float64)
+    M, n_code, dsub = codebooks.shape
+    coarse = centroids @ u_q
+    lut = np.empty((M, n_code), dtype=np.float64)
+    for m in range(M):
+        lut[m] = codebooks[m] @ u_q[m * dsub:(m + 1) * dsub]
+    return coarse, lut
+
+
+# --------------------------------------------------------------------------- O4
+def adc_logits(r_q: float, coarse: np.ndarray, lut: np.ndarray, codes: np.ndarray,
+               list_ids: np.ndarray, key_norms: np.ndarray, sm_scale: float) -> np.ndarray:
+    """Eq. 2: l~_i = (r_q r_i / sqrt d) (u_q.c_{a_i} + sum_m LUT[m][z_im]).
+
+    codes [n, M] uint8, list_ids [n], key_norms [n] (None = all ones).
+    sm_scale is 1/sqrt(d)."""
+    codes = np.asarray(codes).astype(np.int64)
+    list_ids = np.asarray(list_ids).astype(np.int64)
+    n, M = codes.shape
+    s = coarse[list_ids].astype(np.float64)
+    for m in range(M):
+        s = s + lut[m][codes[:, m]]
+    r = np.ones(n) if key_norms is None else np.asarray(key_norms, dtype=np.float64)
+    return (r_q * r * sm_scale) * s
+
+
+# --------------------------------------------------------------------------- O5
+def select_topk(scores: np.ndarray, k: int) -> np.ndarray:
+    """Indices (into `scores`) of the k largest entries; among equal scores the
+    lower index is taken first (Eq. 3 with a stable tie rule)."""
+    if k <= 0:
+        return np.zeros(0, dtype=np.int64)
+    order = np.argsort(-np.asarray(scores, dtype=np.float64), kind="stable")
+    return np.sort(order[:k])
+
+
+# --------------------------------------------------------------------------- paged KV
+def gather_rows(cache_flat: np.ndarray, block_table_row: np.ndarray, positions: np.ndarray,
+                kv_head: int, head_dim: int, page_size: int,
+                stride_page: int, stride_token: int, stride_head: int) -> np.ndarray:
+    """Rows of one KV head at the given sequence positions, read in place from a
+    paged cache described by element strides (Sec. 3.3: the gather reads the
+    engine's pages in place)."""
+    positions = np.asarray(positions, dtype=np.int64)
+    page = np.asarray(block_table_row, dtype=np.int64)[positions // page_size]
+    off = page * stride_page + (positions % page_size) * stride_token + kv_head * stride_head
+    idx = off[:, None] + np.arange(head_dim, dtype=np.int64)[None, :]
+    return np.asarray(cache_flat)[idx].astype(np.float64)
+
+
+# --------------------------------------------------------------------------- O6-O9
+def hybrid_output(q: np.ndarray, keys_E: np.ndarray, vals_E: np.ndarray,
+                  logits_B: np.ndarray, lists_B: np.ndarray, list_vmeans: np.ndarray,
+                  sm_scale: float):
+    """Eq. 4-5 for one query head.
+
+    keys_E, vals_E: original rows of the exact set E.  logits_B, lists_B: the
+    approximate logit and list id of every background token (B = R \\ T).
+    list_vmeans [n_list, d]: stored per-list value means.
+    Returns y^ and a dict with the intermediate sums (all relative to m_0)."""
+    q = np.asarray(q, dtype=np.float64)
+    d = q.shape[0]
+    list_vmeans = np.asarray(list_vmeans, dtype=np.float64)
+    n_list = list_vmeans.shape[0]
+    logits_E = (np.asarray(keys_E, dtype=np.float64).reshape(-1, d) @ q) * sm_scale
+    logits_B = np.asarray(logits_B, dtype=np.float64)
+    lists_B = np.asarray(lists_B).astype(np.int64)
+
+    cands = [x.max() for x in (logits_E, logits_B) if x.size]
+    if not cands:                                   # empty sequence
+        return np.zeros(d), dict(m0=-math.inf, Z_E=0.0, Z_B=0.0, M=np.zeros(n_list),
+                                 logits_E=logits_E)
+    m0 = max(cands)
+    e_E = np.exp(logits_E - m0)
+    e_B = np.exp(logits_B - m0)
+    Z_E = e_E.sum()
+    N_E = e_E @ np.asarray(vals_E, dtype=np.float64).reshape(-1, d)
+    # M_j = sum of e~_i over the background members of list j (empty list -> 0)
+    M_j = np.bincount(lists_B, weights=e_B, minlength=n_list).astype(np.float64)
+    Z_B = M_j.sum()
+    N_B = M_j @ list_vmeans
+    y = (N_E + N_B) / (Z_E + Z_B)
+    return y, dict(m0=m0, Z_E=Z_E, Z_B=Z_B, M=M_j, logits_E=logits_E,
+                   lse=m0 + math.log(Z_E + Z_B))
+
+
+def decode_head(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
+                keys, vals, seq_len, budget_ppm, sm_scale, n_sink=0, n_local=0,
+                round_exact_set_to_page=0):
+    """One (sequence, query head): O1-O9.
+
+    keys / vals are callables position-array -> rows [len, d] (original K, V of the
+    query head's KV head); the index arrays belong to the same KV head and are
+    indexed by sequence position.  Returns a dict with y^ and every intermediate."""
+    q = np.asarray(q, dtype=np.float64)
+    S, L, R = partition(seq_len, n_sink, n_local)
+    k = budget_k(len(R), budget_ppm)
+    if round_exact_set_to_page:
+        total = exact_set_tokens(seq_len, n_sink, n_local, budget_ppm, round_exact_set_to_page)
+        k = min(len(R), total - len(S) - len(L))
+    r_q, u_q = split_query(q)
+    coarse, lut = build_lut(u_q, centroids, codebooks)
+    norms_R = None if key_norms is None else np.asarray(key_norms)[R]
+    approx = adc_logits(r_q, coarse, lut, np.asarray(codes)[R], np.asarray(list_ids)[R],
+                        norms_R, sm_scale)
+    sel_local = select_topk(approx, k)
+    T = R[sel_local]
+    mask_B = np.ones(len(R), dtype=bool)
+    mask_B[sel_local] = False
+    E = np.concatenate([S, L, T])
+    y, aux = hybrid_output(q, keys(E), vals(E), approx[mask_B],
+                           np.asarray(list_ids)[R][mask_B], list_vmeans, sm_scale)
+    kth = float(np.sort(approx)[::-1][k - 1]) if k > 0 else math.nan
+    aux.update(y=y, r_q=r_q, u_q=u_q, coarse=coarse, lut=lut, approx=approx, R=R, T=T,
+               E=E, k=k, kth_score=kth)
+    return aux
+
+
+def decode(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
+           k_cache_flat, v_cache_flat, block_table, seq_lens, *, n_kv_heads, page_size,
+           stride_page, stride_token, stride_head, budget_ppm, sm_scale,
+           n_sink=0, n_local=0, heads=None, batch_items=None):
+    """The whole operator: every (sequence, query head), reading the paged cache in
+    place.  Array layouts are those of the C ABI (q [B,Hq,d]; centroids
+    [B,Hkv,n_list,d]; codebooks [B,Hkv,M,n_code,dsub]; codes [B,Hkv,N_max,M];
+    list_ids / key_norms [B,Hkv,N_max]; list_vmeans [B,Hkv,n_list,d]).
+    Returns {(b, h): decode_head result}; `heads` / `batch_items` restrict the work."""
+    q = np.asarray(q, dtype=np.float64)
+    B, Hq, d = q.shape
+    G = Hq // n_kv_heads
+    out = {}
+    for b in (range(B) if batch_items is None else batch_items):
+        n = int(seq_lens[b])
+        for h in (range(Hq) if heads is None else heads):
+            g = h // G
+            keys = lambda pos, g=g, b=b: gather_rows(k_cache_flat, block_table[b], pos, g, d,
+                                                     page_size, stride_page, stride_token,
+                                                     stride_head)
+            vals = lambda pos, g=g, b=b: gather_rows(v_cache_flat, block_table[b], pos, g, d,
+                                                     page_size, stride_page, stride_token,
+                                                     stride_head)
+            out[(b, h)] = decode_head(
+                q[b, h], centroids[b, g], codebooks[b, g], codes[b, g], list_ids[b, g],
+                None if key_norms is None else key_norms[b, g], list_vmeans[b, g],
+                keys, vals, n, budget_ppm, sm_scale, n_sink, n_local)
+    return out

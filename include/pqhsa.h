@@ -1,0 +1,186 @@
+/*
+ * pqhsa.h -- C ABI of the PQ-HSA decode-step attention operator for NVIDIA B200 (sm_100a).
+ *
+ * The operator (paper Section 3, Eq. 2-5), per sequence b and query head h whose KV head is
+ * g = h / G (G = n_q_heads / n_kv_heads):
+ *
+ *   1. LUT build   coarse[j] = q.c_j and LUT[m][z] = q^(m).p_{m,z}                    (Sec. 3.1)
+ *   2. ADC scan    l~_i = r_i/sqrt(d) * (coarse[a_i] + sum_m LUT[m][z_im]) for every
+ *                  indexed token i, one score row per query head from one pass over the
+ *                  codes of the KV head, plus per-list sums of exp(l~_i - ref)        (Eq. 2, Sec. 3.3)
+ *   3. top-k       T = the k = ceil(rho |R|) tokens with the largest l~_i             (Eq. 3)
+ *   4. hybrid attention: exact logits from the original K rows of T, the approximate
+ *                  logits of all other tokens summed per inverted list and multiplied
+ *                  by the list's stored mean value, one softmax normaliser            (Eq. 4-5)
+ *
+ * (q = r_q u_q, so r_q * (u_q.x) = q.x: the library works with q directly; this is Eq. 2
+ *  with the factor r_q multiplied in.)
+ *
+ * Conventions for every entry point
+ *   - `params` is a HOST pointer.  Every other pointer is a DEVICE pointer owned by the
+ *     caller unless a comment says "host".  The library never allocates, frees or
+ *     synchronises (pqhsa_last_device_status and pqhsa_decode_host excepted), so calls may
+ *     be captured in a CUDA graph.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Arguments are validated on the host first; on error nothing is launched and a
+ *     negative pqhsa_status is returned.  PQHSA_OK (0) means "launched", not "finished".
+ *   - Input arrays are read-only.  Rows past seq_lens[b] are never read.
+ *   - v1 limits: head_dim == 128; pq_ncode == 256 (uint8 codes); pq_m in {8,16,32,64} with
+ *     pq_m * pq_dsub == 128; n_list <= 4096 (and the per-CTA tables must fit shared memory,
+ *     see PQHSA_ERR_UNSUPPORTED); max_seq_len % 4 == 0; page rows 16-byte aligned
+ *     (strides multiples of 8 elements); n_sink == n_local == 0.
+ */
+#ifndef PQHSA_H_
+#define PQHSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PQHSA_OK = 0,
+  PQHSA_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, inconsistent shape      */
+  PQHSA_ERR_UNSUPPORTED = -2,   /* valid request outside the v1 limits above                */
+  PQHSA_ERR_WORKSPACE = -3,     /* ws_bytes smaller than pqhsa_workspace_bytes()            */
+  PQHSA_ERR_CUDA = -4,          /* a CUDA runtime call (launch, memset, copy) failed        */
+  PQHSA_ERR_DEVICE_CHECK = -5   /* a kernel recorded an inconsistency in the status word    */
+} pqhsa_status;
+
+typedef enum { PQHSA_F16 = 0, PQHSA_BF16 = 1 } pqhsa_dtype;
+
+/* Shape of one decode step (host struct).  Notation follows the paper. */
+typedef struct {
+  int32_t batch;              /* B   sequences                                              */
+  int32_t n_q_heads;          /* H_q query heads                                            */
+  int32_t n_kv_heads;         /* H_kv KV heads; G = H_q / H_kv                              */
+  int32_t head_dim;           /* d  (128)                                                   */
+  int32_t n_list;             /* inverted lists per (sequence, KV head)                     */
+  int32_t pq_m;               /* M  PQ subspaces                                            */
+  int32_t pq_dsub;            /* dims per subspace, M * dsub == d                           */
+  int32_t pq_ncode;           /* 2^b codewords per subspace (256)                           */
+  int32_t max_seq_len;        /* N_max: row stride of codes / list_ids / key_norms / scores */
+  int32_t page_size;          /* tokens per KV page                                         */
+  int32_t max_pages_per_seq;  /* row stride of block_table                                  */
+  int32_t n_sink;             /* |S| sink prefix (Sec. 3.2); must be 0 in v1                */
+  int32_t n_local;            /* |L| local window (Sec. 3.2); must be 0 in v1               */
+  uint32_t budget_ppm;        /* rho in parts per million; k_b = ceil(|R_b| * ppm / 1e6),   */
+                              /* computed in 64-bit integers on the device from seq_lens    */
+  int32_t k_max;              /* row stride of sel_idx; >= ceil(max_seq_len * ppm / 1e6)    */
+  float sm_scale;             /* 1/sqrt(d) (Eq. 1)                                          */
+  int32_t dtype;              /* pqhsa_dtype of q, K, V and out                             */
+} pqhsa_params;
+
+/* IVF-PQ index, one per (sequence, KV head) (Sec. 3.1).  Device pointers, read-only. */
+typedef struct {
+  const float* centroids;     /* [B][H_kv][n_list][d]      c_j                              */
+  const float* codebooks;     /* [B][H_kv][M][256][dsub]   p_{m,z}; subspace m = dims       */
+                              /*                           [m*dsub, (m+1)*dsub)             */
+  const uint8_t* codes;       /* [B][H_kv][N_max][M]       z_im                             */
+  const uint16_t* list_ids;   /* [B][H_kv][N_max]          a_i < n_list                     */
+  const float* key_norms;     /* [B][H_kv][N_max]          r_i, or NULL for all ones        */
+  const float* list_vmeans;   /* [B][H_kv][n_list][d]      stored mean value of ALL members */
+                              /*                           of each list (Eq. 4); 0 if empty */
+} pqhsa_index;
+
+/* Engine-owned paged KV cache, read in place through element strides (Sec. 3.3, App. E):
+ * row of (page p, slot t, KV head g) starts at  base + p*stride_page + t*stride_token +
+ * g*stride_head  elements and holds d contiguous elements.  Covers both a split layout
+ * ([page][slot][head][d], K and V separate) and an interleaved one ([page][head][slot][2d],
+ * v_cache = k_cache + d). */
+typedef struct {
+  const void* k_cache;
+  const void* v_cache;
+  int64_t stride_page, stride_token, stride_head;
+  const int32_t* block_table; /* [B][max_pages_per_seq]: page id of the i-th page of b      */
+} pqhsa_paged_kv;
+
+/* Which intermediate buffer pqhsa_buffer_elems() sizes. */
+typedef enum {
+  PQHSA_BUF_LUT = 0,            /* float   [B][H_kv][n_hg][256][M][Gc]                        */
+  PQHSA_BUF_COARSE = 1,         /* float   [B][H_kv][n_hg][n_list][Gc]                        */
+  PQHSA_BUF_SCORES = 2,         /* float   [B][H_q][N_max]                                    */
+  PQHSA_BUF_LIST_PARTIALS = 3,  /* float   [B][H_q][n_part][1 + n_list]                       */
+  PQHSA_BUF_SEL_IDX = 4,        /* int32   [B][H_q][k_max]                                    */
+  PQHSA_BUF_SEL_COUNT = 5,      /* int32   [B][H_q]                                           */
+  PQHSA_BUF_KTH = 6             /* float   [B][H_q]                                           */
+} pqhsa_buffer;
+
+/* Query heads of a group are processed Gc at a time (Gc = G for G <= 2, else 4); a group
+ * has n_hg = ceil(G / Gc) such head groups.  In LUT / COARSE the last index is the head
+ * within its head group; slots past G are zero. */
+int pqhsa_heads_per_group(const pqhsa_params* params);        /* Gc, or <0 on error          */
+int pqhsa_num_partials(const pqhsa_params* params);           /* n_part, or <0 on error      */
+/* Number of ELEMENTS of an intermediate buffer (0 on error). Host-only arithmetic. */
+size_t pqhsa_buffer_elems(const pqhsa_params* params, int which);
+/* Bytes of scratch that any single entry point below needs (pqhsa_decode needs the most:
+ * it also carves every intermediate buffer from it).  256-byte aligned base required. */
+size_t pqhsa_workspace_bytes(const pqhsa_params* params);
+
+/* Step 1 (Sec. 3.1, text after Eq. 2).  q [B][H_q][d] in params->dtype.
+ * Writes lut[..][z][m][g] = sm_scale * q_h^(m).p_{m,z} and
+ * coarse[..][j][g] = sm_scale * q_h.c_j with h = kv*G + hg*Gc + g. */
+int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                    float* lut, float* coarse, void* stream);
+
+/* Step 2 (Eq. 2 and the fused per-list reduction of Sec. 3.3).  seq_lens [B] int32.
+ * Writes scores[b][h][i] = l~_i for i < seq_lens[b], and for every segment s of the row
+ * (a contiguous token range scanned by one CTA; at most n_part per row, the count is a
+ * function of seq_lens only) list_partials[b][h][s][0] = ref_s = max l~_i of the segment
+ * and [1+j] = sum over the segment's members of list j of exp(l~_i - ref_s). */
+int pqhsa_scan(const pqhsa_params* params, const pqhsa_index* index, const float* lut,
+               const float* coarse, const int32_t* seq_lens, float* scores,
+               float* list_partials, void* ws, size_t ws_bytes, void* stream);
+
+/* Step 3 (Eq. 3).  Exact top-k of every score row: sel_idx[b][h][0..k_b) = positions of the
+ * k_b largest scores (order unspecified; equal scores: lower position first),
+ * sel_count[b][h] = k_b, kth_score[b][h] = the k_b-th largest score (NaN if k_b == 0). */
+int pqhsa_select(const pqhsa_params* params, const float* scores, const int32_t* seq_lens,
+                 int32_t* sel_idx, int32_t* sel_count, float* kth_score,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/* Step 4 (Eq. 4-5).  Gathers the selected K/V rows from the paged cache, replaces their
+ * approximate logits by exact ones, takes the selected tokens' mass out of their lists'
+ * sums, folds in the n_list mean-value terms and normalises once.
+ * out [B][H_q][d] in params->dtype; lse_or_null [B][H_q] = log of the normaliser. */
+int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
+                        const pqhsa_index* index, const float* scores,
+                        const float* list_partials, const int32_t* sel_idx,
+                        const int32_t* sel_count, const int32_t* seq_lens, void* out,
+                        float* lse_or_null, void* ws, size_t ws_bytes, void* stream);
+
+/* Steps 1-4 back to back on one stream (Sec. 3.3: the decode step of one layer); all
+ * intermediates live in `ws`. */
+int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                 const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/* pqhsa_decode for a caller whose query and output live in HOST memory (pinned for the
+ * copies to be asynchronous): copies q_host -> q_dev_staging, runs the step, copies
+ * out_dev_staging -> out_host and waits for the stream.  The index, the KV cache and
+ * seq_lens stay resident on the device, as they do in a serving engine. */
+int pqhsa_decode_host(const pqhsa_params* params, const void* q_host, void* q_dev_staging,
+                      const pqhsa_index* index, const pqhsa_paged_kv* kv,
+                      const int32_t* seq_lens, void* out_dev_staging, void* out_host,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/* Reads the status word kernels set when they meet an inconsistency (selected count != k,
+ * seq_len > max_seq_len): copies it to the host and waits for `stream`.  Returns PQHSA_OK
+ * or PQHSA_ERR_DEVICE_CHECK.  Valid after pqhsa_select / pqhsa_decode on the same ws. */
+int pqhsa_last_device_status(const pqhsa_params* params, void* ws, void* stream);
+
+/* Byte offset inside `ws` of an intermediate buffer after pqhsa_decode (for inspection by
+ * tests and tools); (size_t)-1 on error. */
+size_t pqhsa_decode_buffer_offset(const pqhsa_params* params, int which);
+
+/* Number of kernels (memsets included) pqhsa_decode enqueues for these params. */
+int pqhsa_decode_launch_count(const pqhsa_params* params);
+
+const char* pqhsa_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PQHSA_H_ */

@@ -1,0 +1,377 @@
+// Host side of the C ABI: argument validation, launch plan, workspace carve-up and the
+// entry points declared in pqhsa.h.  Nothing here allocates device memory or synchronises,
+// except pqhsa_last_device_status and pqhsa_decode_host, which say so.
+#include <mutex>
+
+#include "common.cuh"
+
+namespace pqhsa {
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr size_t kMaxSmemPerCta = 227 * 1024 - 1024;   // opt-in limit minus static shared memory
+constexpr int kDefaultSms = 148;                        // B200
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+int sm_count() {
+  static int cached[64];
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return kDefaultSms; }
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev < 0 || dev >= 64) return kDefaultSms;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = kDefaultSms;
+    }
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+}  // namespace
+
+int make_plan(const pqhsa_params* p, Plan* pl) {
+  if (p == nullptr || pl == nullptr) return PQHSA_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->head_dim <= 0 ||
+      p->n_list <= 0 || p->pq_m <= 0 || p->pq_dsub <= 0 || p->pq_ncode <= 0 ||
+      p->max_seq_len <= 0 || p->page_size <= 0 || p->max_pages_per_seq <= 0 || p->k_max <= 0 ||
+      p->n_sink < 0 || p->n_local < 0)
+    return PQHSA_ERR_INVALID_ARG;
+  if (p->n_q_heads % p->n_kv_heads != 0) return PQHSA_ERR_INVALID_ARG;
+  if (p->pq_m * p->pq_dsub != p->head_dim) return PQHSA_ERR_INVALID_ARG;
+  if (p->budget_ppm > 1000000u) return PQHSA_ERR_INVALID_ARG;
+  if (p->dtype != PQHSA_F16 && p->dtype != PQHSA_BF16) return PQHSA_ERR_INVALID_ARG;
+  if (!(p->sm_scale > 0.f)) return PQHSA_ERR_INVALID_ARG;
+  if ((long long)p->max_pages_per_seq * p->page_size < p->max_seq_len) return PQHSA_ERR_INVALID_ARG;
+  const long long k_need = ((long long)p->max_seq_len * p->budget_ppm + 999999LL) / 1000000LL;
+  if (p->k_max < k_need) return PQHSA_ERR_INVALID_ARG;
+
+  if (p->head_dim != kHeadDim || p->pq_ncode != kNCode) return PQHSA_ERR_UNSUPPORTED;
+  if (p->pq_m != 8 && p->pq_m != 16 && p->pq_m != 32 && p->pq_m != 64) return PQHSA_ERR_UNSUPPORTED;
+  if (p->n_list > 4096 || p->max_seq_len % 4 != 0) return PQHSA_ERR_UNSUPPORTED;
+  if (p->n_sink != 0 || p->n_local != 0) return PQHSA_ERR_UNSUPPORTED;
+  const int G = p->n_q_heads / p->n_kv_heads;
+  if (G > 16) return PQHSA_ERR_UNSUPPORTED;
+
+  Plan& o = *pl;
+  o.B = p->batch; o.Hq = p->n_q_heads; o.Hkv = p->n_kv_heads; o.G = G;
+  o.Gc = G <= 2 ? G : 4;
+  o.n_hg = (G + o.Gc - 1) / o.Gc;
+  o.n_list = p->n_list; o.M = p->pq_m; o.dsub = p->pq_dsub;
+  o.N_max = p->max_seq_len; o.page_size = p->page_size; o.max_pages = p->max_pages_per_seq;
+  o.k_max = p->k_max; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
+  o.num_sms = sm_count();
+  o.scan_ctas = o.num_sms;
+  o.upb = o.Hkv * o.n_hg;
+  o.n_part = o.scan_ctas / o.upb + 2;
+  o.rows = o.B * o.Hq;
+  if (scan_smem_bytes(o, true) <= kMaxSmemPerCta) o.coarse_in_smem = 1;
+  else if (scan_smem_bytes(o, false) <= kMaxSmemPerCta) o.coarse_in_smem = 0;
+  else return PQHSA_ERR_UNSUPPORTED;
+
+  o.hist_chunks = ceil_div(2LL * o.num_sms, o.rows);
+  const int max_chunks = o.N_max / 4096 > 0 ? o.N_max / 4096 : 1;
+  if (o.hist_chunks > max_chunks) o.hist_chunks = max_chunks;
+  if (o.hist_chunks < 1) o.hist_chunks = 1;
+  o.cand_cap = o.N_max / 4 > 4096 ? o.N_max / 4 : 4096;
+  if (o.cand_cap > o.N_max) o.cand_cap = o.N_max;
+  o.splits = ceil_div(4LL * o.num_sms, o.rows);
+  const int max_splits = (o.k_max + o.n_list / 4) / 32 > 0 ? (o.k_max + o.n_list / 4) / 32 : 1;
+  if (o.splits > max_splits) o.splits = max_splits;
+  if (o.splits > 64) o.splits = 64;
+  if (o.splits < 1) o.splits = 1;
+  return PQHSA_OK;
+}
+
+static size_t buffer_elems(const Plan& pl, int which) {
+  const size_t units = (size_t)pl.B * pl.Hkv * pl.n_hg;
+  switch (which) {
+    case PQHSA_BUF_LUT: return units * kNCode * pl.M * pl.Gc;
+    case PQHSA_BUF_COARSE: return units * pl.n_list * pl.Gc;
+    case PQHSA_BUF_SCORES: return (size_t)pl.rows * pl.N_max;
+    case PQHSA_BUF_LIST_PARTIALS: return (size_t)pl.rows * pl.n_part * (pl.n_list + 1);
+    case PQHSA_BUF_SEL_IDX: return (size_t)pl.rows * pl.k_max;
+    case PQHSA_BUF_SEL_COUNT: return (size_t)pl.rows;
+    case PQHSA_BUF_KTH: return (size_t)pl.rows;
+    default: return 0;
+  }
+}
+
+void make_layout(const Plan& pl, WsLayout* L) {
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  L->zero_begin = o;
+  L->status = take(16);
+  L->hist1 = take((size_t)pl.rows * kHistBins * 4);
+  L->hist2 = take((size_t)pl.rows * kHistBins * 4);
+  L->counters = take((size_t)pl.rows * 16);
+  L->attend_tickets = take((size_t)pl.rows * 4);
+  L->zero_bytes = o - L->zero_begin;
+  L->rowstate = take((size_t)pl.rows * 16);
+  L->cand = take((size_t)pl.rows * pl.cand_cap * 8);
+  L->bg_mass = take((size_t)pl.rows * pl.n_list * 4);
+  L->bg_max = take((size_t)pl.rows * 4);
+  L->split_part = take((size_t)pl.rows * pl.splits * (2 + kHeadDim) * 4);
+  L->stage_end = o;
+  L->lut = take(buffer_elems(pl, PQHSA_BUF_LUT) * 4);
+  L->coarse = take(buffer_elems(pl, PQHSA_BUF_COARSE) * 4);
+  L->scores = take(buffer_elems(pl, PQHSA_BUF_SCORES) * 4);
+  L->list_partials = take(buffer_elems(pl, PQHSA_BUF_LIST_PARTIALS) * 4);
+  L->sel_idx = take(buffer_elems(pl, PQHSA_BUF_SEL_IDX) * 4);
+  L->sel_count = take(buffer_elems(pl, PQHSA_BUF_SEL_COUNT) * 4);
+  L->kth = take(buffer_elems(pl, PQHSA_BUF_KTH) * 4);
+  L->total = o;
+}
+
+}  // namespace pqhsa
+
+using namespace pqhsa;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_index(const pqhsa_index* ix) {
+  if (ix == nullptr || ix->centroids == nullptr || ix->codebooks == nullptr ||
+      ix->codes == nullptr || ix->list_ids == nullptr || ix->list_vmeans == nullptr)
+    return PQHSA_ERR_INVALID_ARG;
+  if (!aligned16(ix->centroids) || !aligned16(ix->codes) || !aligned16(ix->list_vmeans))
+    return PQHSA_ERR_INVALID_ARG;
+  return PQHSA_OK;
+}
+
+int check_kv(const pqhsa_paged_kv* kv) {
+  if (kv == nullptr || kv->k_cache == nullptr || kv->v_cache == nullptr ||
+      kv->block_table == nullptr)
+    return PQHSA_ERR_INVALID_ARG;
+  if (!aligned16(kv->k_cache) || !aligned16(kv->v_cache)) return PQHSA_ERR_INVALID_ARG;
+  if (kv->stride_page < 0 || kv->stride_token < 0 || kv->stride_head < 0)
+    return PQHSA_ERR_INVALID_ARG;
+  if (kv->stride_page % 8 || kv->stride_token % 8 || kv->stride_head % 8)
+    return PQHSA_ERR_UNSUPPORTED;
+  return PQHSA_OK;
+}
+
+int check_ws(const void* ws, size_t ws_bytes, size_t need) {
+  if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PQHSA_ERR_INVALID_ARG;
+  return ws_bytes < need ? PQHSA_ERR_WORKSPACE : PQHSA_OK;
+}
+
+int cuda_status(cudaError_t e) { return e == cudaSuccess ? PQHSA_OK : PQHSA_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+int pqhsa_heads_per_group(const pqhsa_params* params) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  return rc != PQHSA_OK ? rc : pl.Gc;
+}
+
+int pqhsa_num_partials(const pqhsa_params* params) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  return rc != PQHSA_OK ? rc : pl.n_part;
+}
+
+size_t pqhsa_buffer_elems(const pqhsa_params* params, int which) {
+  Plan pl;
+  if (make_plan(params, &pl) != PQHSA_OK) return 0;
+  return buffer_elems(pl, which);
+}
+
+size_t pqhsa_workspace_bytes(const pqhsa_params* params) {
+  Plan pl;
+  if (make_plan(params, &pl) != PQHSA_OK) return 0;
+  WsLayout L;
+  make_layout(pl, &L);
+  return L.total;
+}
+
+size_t pqhsa_decode_buffer_offset(const pqhsa_params* params, int which) {
+  Plan pl;
+  if (make_plan(params, &pl) != PQHSA_OK) return (size_t)-1;
+  WsLayout L;
+  make_layout(pl, &L);
+  switch (which) {
+    case PQHSA_BUF_LUT: return L.lut;
+    case PQHSA_BUF_COARSE: return L.coarse;
+    case PQHSA_BUF_SCORES: return L.scores;
+    case PQHSA_BUF_LIST_PARTIALS: return L.list_partials;
+    case PQHSA_BUF_SEL_IDX: return L.sel_idx;
+    case PQHSA_BUF_SEL_COUNT: return L.sel_count;
+    case PQHSA_BUF_KTH: return L.kth;
+    default: return (size_t)-1;
+  }
+}
+
+int pqhsa_decode_launch_count(const pqhsa_params* params) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  return 7;   // memset, LUT build, scan, select histogram, select filter, background prep, attend
+}
+
+int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                    float* lut, float* coarse, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if ((rc = check_index(index)) != PQHSA_OK) return rc;
+  if (q == nullptr || lut == nullptr || coarse == nullptr || !aligned16(lut) || !aligned16(coarse))
+    return PQHSA_ERR_INVALID_ARG;
+  return cuda_status(launch_build_lut(pl, q, *index, lut, coarse, static_cast<cudaStream_t>(stream)));
+}
+
+int pqhsa_scan(const pqhsa_params* params, const pqhsa_index* index, const float* lut,
+               const float* coarse, const int32_t* seq_lens, float* scores, float* list_partials,
+               void* ws, size_t ws_bytes, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if ((rc = check_index(index)) != PQHSA_OK) return rc;
+  if (lut == nullptr || coarse == nullptr || seq_lens == nullptr || scores == nullptr ||
+      list_partials == nullptr || !aligned16(lut) || !aligned16(coarse) || !aligned16(scores))
+    return PQHSA_ERR_INVALID_ARG;
+  WsLayout L;
+  make_layout(pl, &L);
+  if ((rc = check_ws(ws, ws_bytes, L.stage_end)) != PQHSA_OK) return rc;
+  char* w = static_cast<char*>(ws);
+  return cuda_status(launch_scan(pl, *index, lut, coarse, seq_lens, scores, list_partials,
+                                 reinterpret_cast<int*>(w + L.status),
+                                 static_cast<cudaStream_t>(stream)));
+}
+
+int pqhsa_select(const pqhsa_params* params, const float* scores, const int32_t* seq_lens,
+                 int32_t* sel_idx, int32_t* sel_count, float* kth_score, void* ws,
+                 size_t ws_bytes, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if (scores == nullptr || seq_lens == nullptr || sel_idx == nullptr || sel_count == nullptr ||
+      kth_score == nullptr || !aligned16(scores))
+    return PQHSA_ERR_INVALID_ARG;
+  WsLayout L;
+  make_layout(pl, &L);
+  if ((rc = check_ws(ws, ws_bytes, L.stage_end)) != PQHSA_OK) return rc;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(w + L.zero_begin, 0, L.zero_bytes, st) != cudaSuccess) return PQHSA_ERR_CUDA;
+  return cuda_status(launch_select(pl, L, w, scores, seq_lens, sel_idx, sel_count, kth_score, st));
+}
+
+int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
+                        const pqhsa_index* index, const float* scores, const float* list_partials,
+                        const int32_t* sel_idx, const int32_t* sel_count, const int32_t* seq_lens,
+                        void* out, float* lse_or_null, void* ws, size_t ws_bytes, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if ((rc = check_index(index)) != PQHSA_OK) return rc;
+  if ((rc = check_kv(kv)) != PQHSA_OK) return rc;
+  if (q == nullptr || scores == nullptr || list_partials == nullptr || sel_idx == nullptr ||
+      sel_count == nullptr || seq_lens == nullptr || out == nullptr)
+    return PQHSA_ERR_INVALID_ARG;
+  WsLayout L;
+  make_layout(pl, &L);
+  if ((rc = check_ws(ws, ws_bytes, L.stage_end)) != PQHSA_OK) return rc;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(w + L.attend_tickets, 0, (size_t)pl.rows * 4, st) != cudaSuccess)
+    return PQHSA_ERR_CUDA;
+  return cuda_status(launch_attend(pl, L, w, q, *kv, *index, scores, list_partials, sel_idx,
+                                   sel_count, seq_lens, out, lse_or_null, st));
+}
+
+int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                 const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out, void* ws,
+                 size_t ws_bytes, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if ((rc = check_index(index)) != PQHSA_OK) return rc;
+  if ((rc = check_kv(kv)) != PQHSA_OK) return rc;
+  if (q == nullptr || seq_lens == nullptr || out == nullptr) return PQHSA_ERR_INVALID_ARG;
+  WsLayout L;
+  make_layout(pl, &L);
+  if ((rc = check_ws(ws, ws_bytes, L.total)) != PQHSA_OK) return rc;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* lut = reinterpret_cast<float*>(w + L.lut);
+  float* coarse = reinterpret_cast<float*>(w + L.coarse);
+  float* scores = reinterpret_cast<float*>(w + L.scores);
+  float* partials = reinterpret_cast<float*>(w + L.list_partials);
+  int32_t* sel_idx = reinterpret_cast<int32_t*>(w + L.sel_idx);
+  int32_t* sel_count = reinterpret_cast<int32_t*>(w + L.sel_count);
+  float* kth = reinterpret_cast<float*>(w + L.kth);
+  if (cudaMemsetAsync(w + L.zero_begin, 0, L.zero_bytes, st) != cudaSuccess) return PQHSA_ERR_CUDA;
+  cudaError_t e = launch_build_lut(pl, q, *index, lut, coarse, st);
+  if (e == cudaSuccess)
+    e = launch_scan(pl, *index, lut, coarse, seq_lens, scores, partials,
+                    reinterpret_cast<int*>(w + L.status), st);
+  if (e == cudaSuccess) e = launch_select(pl, L, w, scores, seq_lens, sel_idx, sel_count, kth, st);
+  if (e == cudaSuccess)
+    e = launch_attend(pl, L, w, q, *kv, *index, scores, partials, sel_idx, sel_count, seq_lens,
+                      out, nullptr, st);
+  return cuda_status(e);
+}
+
+int pqhsa_decode_host(const pqhsa_params* params, const void* q_host, void* q_dev_staging,
+                      const pqhsa_index* index, const pqhsa_paged_kv* kv, const int32_t* seq_lens,
+                      void* out_dev_staging, void* out_host, void* ws, size_t ws_bytes,
+                      void* stream) {
+  if (params == nullptr || q_host == nullptr || q_dev_staging == nullptr ||
+      out_dev_staging == nullptr || out_host == nullptr)
+    return PQHSA_ERR_INVALID_ARG;
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)pl.rows * kHeadDim * 2;
+  if (cudaMemcpyAsync(q_dev_staging, q_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return PQHSA_ERR_CUDA;
+  rc = pqhsa_decode(params, q_dev_staging, index, kv, seq_lens, out_dev_staging, ws, ws_bytes,
+                    stream);
+  if (rc != PQHSA_OK) return rc;
+  if (cudaMemcpyAsync(out_host, out_dev_staging, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return PQHSA_ERR_CUDA;
+  return cuda_status(cudaStreamSynchronize(st));
+}
+
+int pqhsa_last_device_status(const pqhsa_params* params, void* ws, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if (ws == nullptr) return PQHSA_ERR_INVALID_ARG;
+  WsLayout L;
+  make_layout(pl, &L);
+  int host = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&host, static_cast<char*>(ws) + L.status, sizeof(int),
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return PQHSA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return PQHSA_ERR_CUDA;
+  return host == 0 ? PQHSA_OK : PQHSA_ERR_DEVICE_CHECK;
+}
+
+const char* pqhsa_status_string(int status) {
+  switch (status) {
+    case PQHSA_OK: return "ok";
+    case PQHSA_ERR_INVALID_ARG: return "invalid argument";
+    case PQHSA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case PQHSA_ERR_WORKSPACE: return "workspace too small";
+    case PQHSA_ERR_CUDA: return "CUDA runtime error";
+    case PQHSA_ERR_DEVICE_CHECK: return "device-side consistency check failed";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,152 @@
+// Shared declarations of the PQ-HSA decode library (host + device).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "pqhsa.h"
+
+namespace pqhsa {
+
+constexpr int kHeadDim = 128;
+constexpr int kNCode = 256;
+constexpr int kTile = 32;            // tokens per scan tile: one token per lane
+constexpr int kScanThreads = 512;
+constexpr int kScanMinTiles = kScanThreads / 32;   // a scan CTA gets at least one tile per warp
+constexpr int kHistBins = 4096;      // 12-bit radix digits for the two coarse select levels
+constexpr int kSelThreads = 512;
+constexpr int kAttendThreads = 128;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegligibleLog2 = -64.0f;   // exp2 arguments below this add nothing to a sum
+
+// Host-derived launch plan; passed by value to kernels.
+struct Plan {
+  int B, Hq, Hkv, G, Gc, n_hg;       // Gc heads per scan pass, n_hg = ceil(G / Gc)
+  int n_list, M, dsub;
+  int N_max, page_size, max_pages;
+  int k_max;
+  uint32_t ppm;
+  float sm_scale;
+  int dtype;
+  int scan_ctas;                     // P: persistent scan CTAs (= number of SMs)
+  int n_part;                        // list-partial slots per score row
+  int upb;                           // scan units per sequence = Hkv * n_hg
+  int rows;                          // B * Hq score rows
+  int hist_chunks;                   // CTAs per row in the select kernels
+  int cand_cap;                      // candidate slots per row
+  int splits;                        // split-K CTAs per row in the attend kernel
+  int coarse_in_smem;                // scan keeps the coarse table in shared memory
+  int num_sms;
+};
+
+// Workspace carve-up (byte offsets from a 256-byte aligned base).
+struct WsLayout {
+  size_t status;                     // int32[4]: device status word (+ padding)
+  size_t zero_begin, zero_bytes;     // region cleared by one memset before select
+  size_t hist1, hist2;               // uint32 [rows][kHistBins] each
+  size_t counters;                   // uint32 [rows][4]: ticket1, ticket2, n_out, n_cand
+  size_t attend_tickets;             // uint32 [rows]
+  size_t rowstate;                   // int32  [rows][4]: b1, k1, k, n
+  size_t cand;                       // uint2  [rows][cand_cap]: (key, position)
+  size_t bg_mass;                    // float  [rows][n_list]: M_j relative to bg_max
+  size_t bg_max;                     // float  [rows]
+  size_t split_part;                 // float  [rows][splits][2 + 128]: m, Z, N[128]
+  size_t stage_end;                  // end of what a single stage call needs
+  // intermediates of the fused entry point
+  size_t lut, coarse, scores, list_partials, sel_idx, sel_count, kth;
+  size_t total;
+};
+
+int make_plan(const pqhsa_params* p, Plan* plan);          // returns pqhsa_status
+void make_layout(const Plan& plan, WsLayout* L);
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint32_t score_key(float s) {
+  // Order-preserving map float -> uint32 (larger score <-> larger key); -0 and +0 coincide.
+  uint32_t u = __float_as_uint(s + 0.0f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_score(uint32_t k) {
+  uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+  return __uint_as_float(u);
+}
+
+// k_b = ceil(n * ppm / 1e6) in 64-bit integers, clipped to n (Eq. 3).
+__device__ __forceinline__ int budget_k(int n, uint32_t ppm) {
+  if (n <= 0) return 0;
+  long long k = ((long long)n * (long long)ppm + 999999LL) / 1000000LL;
+  return (int)(k < (long long)n ? k : (long long)n);
+}
+
+__device__ __forceinline__ int clamp_len(int n, int n_max) {
+  return n < 0 ? 0 : (n > n_max ? n_max : n);
+}
+
+// The scan walks one global sequence of 32-token tiles: sequence-major, then the
+// H_kv * n_hg units (KV head, head group) of the sequence, then the tiles of the unit.
+// CTA c of P_eff owns tiles [c*T/P_eff, (c+1)*T/P_eff).  Producer (scan) and consumer
+// (background preparation) both derive the same split from seq_lens alone.
+struct ScanSplit {
+  long long T;       // total tiles
+  int P_eff;         // CTAs that take part
+};
+__device__ __forceinline__ int seq_tiles(const int32_t* seq_lens, int b, int n_max) {
+  return (clamp_len(seq_lens[b], n_max) + kTile - 1) / kTile;
+}
+__device__ __forceinline__ ScanSplit scan_split(const int32_t* seq_lens, int B, int n_max,
+                                                int upb, int P) {
+  long long T = 0;
+  for (int b = 0; b < B; ++b) T += (long long)seq_tiles(seq_lens, b, n_max) * upb;
+  long long pe = T / kScanMinTiles;
+  if (pe < 1) pe = 1;
+  if (pe > P) pe = P;
+  return ScanSplit{T, (int)pe};
+}
+__device__ __forceinline__ long long split_start(const ScanSplit& s, int c) {
+  return (long long)c * s.T / s.P_eff;
+}
+__device__ __forceinline__ int split_cta_of(const ScanSplit& s, long long tile) {
+  int c = (int)(tile * s.P_eff / s.T);
+  if (c + 1 < s.P_eff && split_start(s, c + 1) <= tile) ++c;
+  return c;
+}
+
+// 2^x by the SFU (ex2.approx): about 2 ulp, flushes results below 2^-126 to zero.
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ------------------------------------------------------------------ stage launchers
+// Each returns a cudaError_t from the launch (cudaSuccess if nothing had to run).
+cudaError_t launch_build_lut(const Plan& pl, const void* q, const pqhsa_index& ix, float* lut,
+                             float* coarse, cudaStream_t st);
+cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,
+                        const float* coarse, const int32_t* seq_lens, float* scores,
+                        float* list_partials, int* status, cudaStream_t st);
+cudaError_t launch_select(const Plan& pl, const WsLayout& L, char* ws, const float* scores,
+                          const int32_t* seq_lens, int32_t* sel_idx, int32_t* sel_count,
+                          float* kth, cudaStream_t st);
+cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const void* q,
+                          const pqhsa_paged_kv& kv, const pqhsa_index& ix, const float* scores,
+                          const float* list_partials, const int32_t* sel_idx,
+                          const int32_t* sel_count, const int32_t* seq_lens, void* out,
+                          float* lse, cudaStream_t st);
+size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem);
+
+}  // namespace pqhsa

@@ -117,7 +117,7 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
     dev = inp.q.device
     B, Hkv, d = cfg.batch, cfg.n_kv_heads, cfg.head_dim
     M, dsub, nl, nc = cfg.pq_m, cfg.pq_dsub, cfg.n_list, cfg.pq_ncode
-    Nmax = max(cfg.max_seq_len, 1)
+    Nmax = max(16, (cfg.max_seq_len + 15) // 16 * 16)   # row stride, padded to whole pages
     out = IvfPqIndex(
         torch.zeros((B, Hkv, nl, d), dtype=torch.float32, device=dev),
         torch.zeros((B, Hkv, M, nc, dsub), dtype=torch.float32, device=dev),

@@ -1,0 +1,209 @@
+"""ctypes binding of libpqhsa.so: same entry points as include/pqhsa.h, argument marshalling only.
+
+Every step of the decode path runs in the library's CUDA kernels.  PyTorch appears here
+only as the owner of device memory and streams.  There is no fallback: if the shared
+library is missing or a call fails, a ``PqhsaError`` is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpqhsa.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_CHECK = 0, -1, -2, -3, -4, -5
+F16, BF16 = 0, 1
+BUF_LUT, BUF_COARSE, BUF_SCORES, BUF_LIST_PARTIALS, BUF_SEL_IDX, BUF_SEL_COUNT, BUF_KTH = range(7)
+
+EXPORTS = [
+    "pqhsa_heads_per_group", "pqhsa_num_partials", "pqhsa_buffer_elems", "pqhsa_workspace_bytes",
+    "pqhsa_build_lut", "pqhsa_scan", "pqhsa_select", "pqhsa_hybrid_attend", "pqhsa_decode",
+    "pqhsa_decode_host", "pqhsa_last_device_status", "pqhsa_decode_buffer_offset",
+    "pqhsa_decode_launch_count", "pqhsa_status_string",
+]
+
+
+class PqhsaError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {status_string(status)} ({status})")
+
+
+class Params(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "batch", "n_q_heads", "n_kv_heads", "head_dim", "n_list", "pq_m", "pq_dsub", "pq_ncode",
+        "max_seq_len", "page_size", "max_pages_per_seq", "n_sink", "n_local")] + [
+        ("budget_ppm", ctypes.c_uint32), ("k_max", ctypes.c_int32), ("sm_scale", ctypes.c_float),
+        ("dtype", ctypes.c_int32)]
+
+
+class Index(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in (
+        "centroids", "codebooks", "codes", "list_ids", "key_norms", "list_vmeans")]
+
+
+class PagedKV(ctypes.Structure):
+    _fields_ = [("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+                ("stride_page", ctypes.c_int64), ("stride_token", ctypes.c_int64),
+                ("stride_head", ctypes.c_int64), ("block_table", ctypes.c_void_p)]
+
+
+_lib_handle = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library.  Raises if it has not been built."""
+    global _lib_handle
+    if _lib_handle is None:
+        if not os.path.exists(LIB_PATH):
+            raise PqhsaError(f"loading {LIB_PATH} (build it with "
+                             "`python -m paper_2609_33746_b200.build`)", ERR_CUDA)
+        L = ctypes.CDLL(LIB_PATH)
+        P, V, Z, I = ctypes.POINTER(Params), ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        PI, PK = ctypes.POINTER(Index), ctypes.POINTER(PagedKV)
+        sig = {
+            "pqhsa_heads_per_group": (I, [P]),
+            "pqhsa_num_partials": (I, [P]),
+            "pqhsa_buffer_elems": (Z, [P, I]),
+            "pqhsa_workspace_bytes": (Z, [P]),
+            "pqhsa_build_lut": (I, [P, V, PI, V, V, V]),
+            "pqhsa_scan": (I, [P, PI, V, V, V, V, V, V, Z, V]),
+            "pqhsa_select": (I, [P, V, V, V, V, V, V, Z, V]),
+            "pqhsa_hybrid_attend": (I, [P, V, PK, PI, V, V, V, V, V, V, V, V, Z, V]),
+            "pqhsa_decode": (I, [P, V, PI, PK, V, V, V, Z, V]),
+            "pqhsa_decode_host": (I, [P, V, V, PI, PK, V, V, V, V, Z, V]),
+            "pqhsa_last_device_status": (I, [P, V, V]),
+            "pqhsa_decode_buffer_offset": (Z, [P, I]),
+            "pqhsa_decode_launch_count": (I, [P]),
+            "pqhsa_status_string": (ctypes.c_char_p, [I]),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib_handle = L
+    return _lib_handle
+
+
+def status_string(status: int) -> str:
+    try:
+        return lib().pqhsa_status_string(int(status)).decode()
+    except PqhsaError:
+        return "library not loaded"
+
+
+def _check(fn: str, status: int) -> None:
+    if status != OK:
+        raise PqhsaError(fn, status)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_pages_per_seq,
+                budget_ppm, dtype, head_dim=128, pq_ncode=256, page_size=16, n_sink=0, n_local=0,
+                k_max=None, sm_scale=None) -> Params:
+    if k_max is None:
+        k_max = max(1, (max_seq_len * budget_ppm + 999_999) // 1_000_000)
+    if sm_scale is None:
+        sm_scale = 1.0 / math.sqrt(head_dim)
+    code = {"fp16": F16, "bf16": BF16, torch.float16: F16, torch.bfloat16: BF16}[dtype]
+    return Params(batch, n_q_heads, n_kv_heads, head_dim, n_list, pq_m, head_dim // pq_m, pq_ncode,
+                  max_seq_len, page_size, max_pages_per_seq, n_sink, n_local, budget_ppm, k_max,
+                  sm_scale, code)
+
+
+def make_index(centroids, codebooks, codes, list_ids, key_norms, list_vmeans) -> Index:
+    return Index(_ptr(centroids), _ptr(codebooks), _ptr(codes), _ptr(list_ids), _ptr(key_norms),
+                 _ptr(list_vmeans))
+
+
+def make_paged_kv(k_cache, v_cache, stride_page, stride_token, stride_head, block_table) -> PagedKV:
+    return PagedKV(_ptr(k_cache), _ptr(v_cache), stride_page, stride_token, stride_head,
+                   _ptr(block_table))
+
+
+# ------------------------------------------------------------------ host-only arithmetic
+def heads_per_group(params: Params) -> int:
+    r = lib().pqhsa_heads_per_group(ctypes.byref(params))
+    _check("pqhsa_heads_per_group", min(r, 0))
+    return r
+
+
+def num_partials(params: Params) -> int:
+    r = lib().pqhsa_num_partials(ctypes.byref(params))
+    _check("pqhsa_num_partials", min(r, 0))
+    return r
+
+
+def buffer_elems(params: Params, which: int) -> int:
+    return lib().pqhsa_buffer_elems(ctypes.byref(params), which)
+
+
+def workspace_bytes(params: Params) -> int:
+    return lib().pqhsa_workspace_bytes(ctypes.byref(params))
+
+
+def decode_buffer_offset(params: Params, which: int) -> int:
+    return lib().pqhsa_decode_buffer_offset(ctypes.byref(params), which)
+
+
+def decode_launch_count(params: Params) -> int:
+    return lib().pqhsa_decode_launch_count(ctypes.byref(params))
+
+
+# ------------------------------------------------------------------ entry points
+def build_lut(params, q, index: Index, lut, coarse, stream=None) -> None:
+    _check("pqhsa_build_lut", lib().pqhsa_build_lut(
+        ctypes.byref(params), _ptr(q), ctypes.byref(index), _ptr(lut), _ptr(coarse),
+        _stream(stream)))
+
+
+def scan(params, index: Index, lut, coarse, seq_lens, scores, list_partials, ws, stream=None) -> None:
+    _check("pqhsa_scan", lib().pqhsa_scan(
+        ctypes.byref(params), ctypes.byref(index), _ptr(lut), _ptr(coarse), _ptr(seq_lens),
+        _ptr(scores), _ptr(list_partials), _ptr(ws), ws.numel() * ws.element_size(),
+        _stream(stream)))
+
+
+def select(params, scores, seq_lens, sel_idx, sel_count, kth_score, ws, stream=None) -> None:
+    _check("pqhsa_select", lib().pqhsa_select(
+        ctypes.byref(params), _ptr(scores), _ptr(seq_lens), _ptr(sel_idx), _ptr(sel_count),
+        _ptr(kth_score), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def hybrid_attend(params, q, kv: PagedKV, index: Index, scores, list_partials, sel_idx, sel_count,
+                  seq_lens, out, lse, ws, stream=None) -> None:
+    _check("pqhsa_hybrid_attend", lib().pqhsa_hybrid_attend(
+        ctypes.byref(params), _ptr(q), ctypes.byref(kv), ctypes.byref(index), _ptr(scores),
+        _ptr(list_partials), _ptr(sel_idx), _ptr(sel_count), _ptr(seq_lens), _ptr(out), _ptr(lse),
+        _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def decode(params, q, index: Index, kv: PagedKV, seq_lens, out, ws, stream=None) -> None:
+    _check("pqhsa_decode", lib().pqhsa_decode(
+        ctypes.byref(params), _ptr(q), ctypes.byref(index), ctypes.byref(kv), _ptr(seq_lens),
+        _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def decode_host(params, q_host, q_staging, index: Index, kv: PagedKV, seq_lens, out_staging,
+                out_host, ws, stream=None) -> None:
+    _check("pqhsa_decode_host", lib().pqhsa_decode_host(
+        ctypes.byref(params), _ptr(q_host), _ptr(q_staging), ctypes.byref(index),
+        ctypes.byref(kv), _ptr(seq_lens), _ptr(out_staging), _ptr(out_host), _ptr(ws),
+        ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def last_device_status(params, ws, stream=None) -> int:
+    return lib().pqhsa_last_device_status(ctypes.byref(params), _ptr(ws), _stream(stream))

@@ -1,0 +1,59 @@
+"""Shared test plumbing: build a workload + index, and hand the same arrays to the oracle."""
+import math
+
+import numpy as np
+import torch
+
+from oracle import pqhsa_oracle as O
+from paper_2609_33746_b200.index_builder import build_index
+from paper_2609_33746_b200.workload import DecodeConfig, generate
+
+
+def make_case(cfg: DecodeConfig, device="cpu"):
+    inp = generate(cfg, device=device)
+    idx = build_index(inp)
+    return inp, idx
+
+
+def oracle_arrays(inp, idx):
+    """numpy views of the inputs in the oracle's (= the C ABI's) layouts, values in float64
+    where they are floating point."""
+    f64 = lambda t: t.detach().cpu().double().numpy()
+    a = dict(
+        q=f64(inp.q), centroids=f64(idx.centroids), codebooks=f64(idx.codebooks),
+        codes=idx.codes.cpu().numpy(), list_ids=idx.list_ids.cpu().numpy().view(np.uint16),
+        key_norms=f64(idx.key_norms), list_vmeans=f64(idx.list_vmeans),
+        k_cache_flat=f64(inp.k_cache.reshape(-1)), v_cache_flat=f64(inp.v_cache.reshape(-1)),
+        block_table=inp.block_table.cpu().numpy(), seq_lens=inp.seq_lens.cpu().numpy())
+    return a
+
+
+def run_oracle(inp, idx, budget_ppm=None, heads=None, batch_items=None, arrays=None):
+    cfg = inp.cfg
+    a = arrays or oracle_arrays(inp, idx)
+    return O.decode(a["q"], a["centroids"], a["codebooks"], a["codes"], a["list_ids"],
+                    a["key_norms"], a["list_vmeans"], a["k_cache_flat"], a["v_cache_flat"],
+                    a["block_table"], a["seq_lens"], n_kv_heads=cfg.n_kv_heads,
+                    page_size=cfg.page_size, stride_page=inp.stride_page,
+                    stride_token=inp.stride_token, stride_head=inp.stride_head,
+                    budget_ppm=cfg.budget_ppm if budget_ppm is None else budget_ppm,
+                    sm_scale=1.0 / math.sqrt(cfg.head_dim), heads=heads, batch_items=batch_items)
+
+
+def selection_matches(gpu_sel, ref, tol=1e-3):
+    """Selected sets are equal except for tokens whose approximate logit is within
+    tol * max(1, |s_k|) of the k-th score s_k; the set size must be exactly k."""
+    gpu = set(int(x) for x in gpu_sel)
+    want = set(int(x) for x in ref["T"])
+    if len(gpu) != ref["k"] or len(gpu_sel) != ref["k"]:
+        return False, f"size {len(gpu_sel)} (unique {len(gpu)}) != k {ref['k']}"
+    if ref["k"] == 0:
+        return True, ""
+    sk = ref["kth_score"]
+    band = tol * max(1.0, abs(sk))
+    approx = ref["approx"]
+    r0 = int(ref["R"][0]) if len(ref["R"]) else 0
+    for i in gpu ^ want:
+        if abs(approx[i - r0] - sk) > band:
+            return False, f"token {i} (score {approx[i - r0]}, kth {sk}) differs outside the tie band"
+    return True, ""

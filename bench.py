@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the PQ-HSA decode-step attention operator on B200.
+
+One "step" = one pqhsa_decode call (LUT build, ADC scan with fused per-list sums, top-k,
+hybrid attention) over one batch of synthetic sequences whose index and paged KV cache are
+resident in HBM.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3_b8_r1] [--impl reference]
+
+Under torchrun (N > 1) every rank runs the same workload on its own GPU with its own seed
+(the operator shards over sequences with no exchange step): weak scaling, value = the sum
+over ranks of algorithmic bytes / max-over-ranks step time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+METRIC = ("decode-attention achieved HBM GB/s at 128K context "
+          "(algorithmic bytes per step / device time per step; us/step = 1000*ms_per_step)")
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+L2_FLUSH_BYTES = 512 << 20
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------ algorithmic bytes
+def algorithmic_bytes(cfg, seq_lens, budget_ppm):
+    """Bytes one step must move ("Algorithmic bytes").  Per sequence and KV head:
+    codes M + norm 4 + list id 2 per token; one score row per query head written once and
+    read once (4+4 B per token per query head); k exact K and V rows of 2*d*2 B per query
+    head plus 64 B for the two 32-byte sectors that return the token's score and list id;
+    one centroid row and one value-mean row (4*d B each) per list; the codebooks once;
+    the lookup table written and read once."""
+    d, M, G = cfg.head_dim, cfg.pq_m, cfg.group
+    total = scan = select = attend = lut = 0
+    for n in seq_lens:
+        k = min(n, (n * budget_ppm + 999_999) // 1_000_000) if n else 0
+        lut_b = cfg.n_list * 4 * d + M * 256 * cfg.pq_dsub * 4 + G * M * 256 * 4 + G * cfg.n_list * 4
+        scan_b = n * (M + 4 + 2) + G * n * 4 + G * M * 256 * 4 + G * cfg.n_list * 4
+        sel_b = G * n * 4 + G * k * 4
+        att_b = G * k * (2 * d * 2 + 64) + cfg.n_list * 4 * d + G * d * 2 * 2
+        lut += cfg.n_kv_heads * lut_b
+        scan += cfg.n_kv_heads * scan_b
+        select += cfg.n_kv_heads * sel_b
+        attend += cfg.n_kv_heads * att_b
+    total = lut + scan + select + attend
+    return dict(total=total, lut=lut, scan=scan, select=select, attend=attend)
+
+
+def dense_attention_bytes(cfg, seq_lens):
+    return sum(cfg.n_kv_heads * n * 2 * cfg.head_dim * 2 for n in seq_lens)
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.thread = [], None, None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        def pump():
+            for line in self.proc.stdout:
+                self.rows.append([x.strip() for x in line.split(",")])
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, pw = [], [], set(), []
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None,
+                    sm_max_mhz=max(mx) if mx else None,
+                    power_w_max=max(pw) if pw else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+# ------------------------------------------------------------------ oracle (CPU baseline / reference arm)
+def oracle_arrays_seq0(inp, idx):
+    """Float64 host copies of what the oracle needs for sequence 0: its index arrays and
+    its own KV pages, re-packed contiguously with an identity block table (a re-layout of
+    inputs; the oracle still reads rows through block table and strides)."""
+    import numpy as np
+    import torch
+    cfg = inp.cfg
+    assert cfg.kv_layout == "split"
+    f64 = lambda t: t.detach().cpu().double().numpy()
+    n = int(inp.seq_lens[0])
+    n_pages = max(1, (n + cfg.page_size - 1) // cfg.page_size)
+    pages = inp.block_table[0, :n_pages].long()
+    return dict(
+        q=f64(inp.q[:1]), centroids=f64(idx.centroids[:1]), codebooks=f64(idx.codebooks[:1]),
+        codes=idx.codes[:1].cpu().numpy(), list_ids=idx.list_ids[:1].cpu().numpy().view(np.uint16),
+        key_norms=f64(idx.key_norms[:1]), list_vmeans=f64(idx.list_vmeans[:1]),
+        k_cache_flat=f64(inp.k_cache[pages].reshape(-1)),
+        v_cache_flat=f64(inp.v_cache[pages].reshape(-1)),
+        block_table=np.arange(n_pages, dtype=np.int32)[None, :],
+        seq_lens=inp.seq_lens[:1].cpu().numpy())
+
+
+def oracle_sample(inp, arrays, cfg, budget_ppm, n_heads):
+    """Runs the float64 oracle, as it stands, on sequence 0 and its first n_heads query heads.
+    Returns (seconds, algorithmic bytes of that sample)."""
+    from helpers import run_oracle
+    t0 = time.perf_counter()
+    run_oracle(inp, None, budget_ppm=budget_ppm, heads=list(range(n_heads)), batch_items=[0],
+               arrays=arrays)
+    dt = time.perf_counter() - t0
+    n = int(arrays["seq_lens"][0])
+    frac = n_heads / cfg.n_q_heads
+    return dt, algorithmic_bytes(cfg, [n], budget_ppm)["total"] * frac
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        n = 1
+    return n
+
+
+# ------------------------------------------------------------------ main
+def parse_workload(name):
+    from paper_2609_33746_b200.workload import named_config
+    return named_config(name)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c3_b8_r1",
+                    help="c3_b{1,8}_r{1,2} (128K, headline), c2, c4, c5_n{16..512}_b{1,32}")
+    ap.add_argument("--impl", default="pqhsa", choices=["pqhsa", "reference"])
+    ap.add_argument("--kmeans-iters", type=int, default=4,
+                    help="Lloyd iterations of the synthetic index (timing does not depend on it)")
+    ap.add_argument("--no-variants", action="store_true",
+                    help="skip the extra c3 variants (B=1, 2%%) reported beside the headline")
+    ap.add_argument("--oracle-heads", type=int, default=8,
+                    help="query heads of sequence 0 the CPU baseline runs")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference" and rank != 0:
+        return 0
+
+    import torch
+    import dataclasses
+    from paper_2609_33746_b200.index_builder import build_index
+    from paper_2609_33746_b200.workload import generate
+
+    if args.impl == "reference":
+        # The oracle arm needs sequence 0 only (same seeds, hence the same keys, values,
+        # queries and index as sequence 0 of the CUDA arm's workload).
+        cfg = parse_workload(args.workload)
+        cfg = dataclasses.replace(cfg, batch=1, seq_lens=cfg.seq_lens[:1],
+                                  kmeans_iters=args.kmeans_iters)
+        dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+        inp = generate(cfg, device=dev)
+        idx = build_index(inp)
+        arrays = oracle_arrays_seq0(inp, idx)
+        heads = max(1, min(args.oracle_heads, cfg.n_q_heads))
+        for _ in range(min(args.warmup, 1)):
+            oracle_sample(inp, arrays, cfg, cfg.budget_ppm, heads)
+        times, nbytes = [], 0
+        for _ in range(args.steps):
+            dt, nbytes = oracle_sample(inp, arrays, cfg, cfg.budget_ppm, heads)
+            times.append(dt)
+        ms = 1000.0 * sum(times) / len(times)
+        val = nbytes / (ms * 1e-3) / 1e9
+        full = parse_workload(args.workload)
+        sample = (f"each step = float64 numpy oracle on sequence 0, query heads 0..{heads - 1} of "
+                  f"{cfg.n_q_heads} ({heads / cfg.n_q_heads / full.batch:.4f} of the workload's step)")
+        line = dict(impl="reference", metric=METRIC, value=val, unit="GB/s", n_gpus=args.gpus,
+                    steps=args.steps, warmup=args.warmup, ms_per_step=ms, higher_is_better=True,
+                    scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                    config=dict(workload=full.name, batch=full.batch, context=full.max_seq_len,
+                                budget_ppm=full.budget_ppm, sample=sample),
+                    cpu_baseline=dict(value=val, unit="GB/s", cores=cpu_threads(), kind="oracle",
+                                      sample=sample, host_cpus=os.cpu_count()),
+                    e2e=dict(value=val, unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+        print(json.dumps(line))
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1 and args.impl != "reference":
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg = parse_workload(args.workload)
+    cfg = dataclasses.replace(cfg, kmeans_iters=args.kmeans_iters, seed=cfg.seed + 97 * rank)
+    t_gen = time.perf_counter()
+    inp = generate(cfg, device=dev)
+    idx = build_index(inp)
+    torch.cuda.synchronize()
+    t_gen = time.perf_counter() - t_gen
+    seq_lens = list(cfg.seq_lens)
+
+    # ---------------------------------------------------------------- our arm
+    from paper_2609_33746_b200 import pqhsa
+    from paper_2609_33746_b200.runner import DecodeOp
+
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def time_decode(op, steps, warmup, staged_events=False):
+        """Per-step device times (ms) of pqhsa_decode with an L2 flush between steps.
+        With staged_events, also per-stage times from pqhsa_decode_events."""
+        for _ in range(warmup):
+            flush.zero_()
+            op.decode()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5 if staged_events else 2)]
+              for _ in range(steps)]
+        if staged_events:
+            for row in ev:
+                for e in row:
+                    e.record()
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(steps):
+            flush.zero_()
+            if staged_events:
+                pqhsa.decode_events(op.params, op.q, op.index, op.kv, op.seq_lens, op.out, op.ws,
+                                    ev[i])
+            else:
+                ev[i][0].record()
+                op.decode()
+                ev[i][1].record()
+        barrier()
+        wall = time.perf_counter() - t0
+        if staged_events:
+            stages = [[row[j].elapsed_time(row[j + 1]) for j in range(4)] for row in ev]
+            return [sum(s) for s in stages], stages, wall
+        return [a.elapsed_time(b) for a, b in ev], None, wall
+
+    def reduce_max(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def measure(op, cfg_v, ppm, steps, warmup, lens):
+        times, _, _ = time_decode(op, steps, warmup)
+        ms = reduce_max(sum(times) / len(times))
+        ab = algorithmic_bytes(cfg_v, lens, ppm)
+        gbs = world * ab["total"] / (ms * 1e-3) / 1e9
+        srt = sorted(times)
+        return dict(ms=ms, gbs=gbs, bytes=ab, p10=srt[len(srt) // 10], p50=srt[len(srt) // 2],
+                    p90=srt[(9 * len(srt)) // 10])
+
+    try:
+        gpu_index = int(os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")[local_rank])
+    except Exception:
+        gpu_index = local_rank
+    sampler = ClockSampler(gpu_index)
+    op = DecodeOp(inp, idx, device=dev)
+    op.decode()
+    torch.cuda.synchronize()
+    assert op.device_status() == pqhsa.OK
+
+    sampler.start()
+    head = measure(op, cfg, cfg.budget_ppm, args.steps, args.warmup, seq_lens)
+    clocks = sampler.stop()
+    launches = args.steps * pqhsa.decode_launch_count(op.params)
+
+    # per-stage times of the same call, recorded by the library around its own stages
+    _, stages, _ = time_decode(op, args.steps, 2, staged_events=True)
+    stage_ms = [statistics.mean(s[j] for s in stages) for j in range(4)]
+    peak, peak_src = measured_peak()
+    scan_bytes = head["bytes"]["scan"]
+    scan_gbs = scan_bytes / (stage_ms[1] * 1e-3) / 1e9
+    roofline = dict(bound="hbm", kernel="scan_kernel (ADC scan + fused per-list sums)",
+                    achieved=scan_gbs, peak=peak, unit="GB/s", frac=scan_gbs / peak,
+                    peak_source=peak_src, traffic=None,
+                    algorithmic_bytes_per_launch=scan_bytes, avg_launch_ms=stage_ms[1],
+                    co_bound="shared-memory LSU: 16 B of table reads per (token, subspace)",
+                    stage_ms=dict(lut=stage_ms[0], scan=stage_ms[1], select=stage_ms[2],
+                                  attend=stage_ms[3]),
+                    whole_step_frac_of_peak=head["gbs"] / world / peak)
+
+    # end to end through the host-buffer entry point: q from pinned host memory, out back
+    q_host = op.q.cpu().pin_memory()
+    out_host = torch.empty_like(q_host).pin_memory()
+    q_stage, out_stage = torch.empty_like(op.q), torch.empty_like(op.q)
+    for _ in range(3):
+        pqhsa.decode_host(op.params, q_host, q_stage, op.index, op.kv, op.seq_lens, out_stage,
+                          out_host, op.ws)
+    barrier()
+    e2e_times = []
+    for _ in range(args.steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        pqhsa.decode_host(op.params, q_host, q_stage, op.index, op.kv, op.seq_lens, out_stage,
+                          out_host, op.ws)
+        e2e_times.append(time.perf_counter() - t0)
+    barrier()
+    e2e_ms = reduce_max(1000.0 * sum(e2e_times) / len(e2e_times))
+    qbytes = op.q.numel() * op.q.element_size()
+    e2e = dict(value=world * head["bytes"]["total"] / (e2e_ms * 1e-3) / 1e9, unit="GB/s",
+               ms_per_step=e2e_ms, h2d_bytes_per_step=qbytes, d2h_bytes_per_step=qbytes,
+               note="pqhsa_decode_host: q from pinned host memory, output read back, stream "
+                    "synchronised, host wall clock; index and paged KV cache stay resident in HBM")
+
+    # the other c3 variants (same tensors: batch 1 = sequence 0, 2% = another budget)
+    variants = {}
+    if cfg.name.startswith("c3") and not args.no_variants:
+        for vb, vp in ((1, 10000), (1, 20000), (8, 10000), (8, 20000)):
+            if vb > cfg.batch or (vb == cfg.batch and vp == cfg.budget_ppm):
+                continue
+            cfg_v = dataclasses.replace(cfg, batch=vb, seq_lens=cfg.seq_lens[:vb], budget_ppm=vp)
+            inp_v = dataclasses.replace(inp, cfg=cfg_v)
+            op_v = DecodeOp(inp_v, idx, device=dev, budget_ppm=vp)
+            r = measure(op_v, cfg_v, vp, args.steps, args.warmup, list(cfg_v.seq_lens))
+            variants[f"c3_b{vb}_r{vp // 10000}"] = dict(
+                us_per_step=1000 * r["ms"], us_p10=1000 * r["p10"], us_p90=1000 * r["p90"],
+                achieved_gbs=r["gbs"] / world, pct_of_8TBps=100 * r["gbs"] / world / NOMINAL_HBM_GBS,
+                algorithmic_mb=r["bytes"]["total"] / 1e6)
+            del op_v
+
+    cpu_baseline = None
+    if rank == 0 and world == 1:
+        heads = max(1, min(args.oracle_heads, cfg.n_q_heads))
+        dt, nbytes = oracle_sample(inp, oracle_arrays_seq0(inp, idx), cfg, cfg.budget_ppm, heads)
+        cpu_baseline = dict(value=nbytes / dt / 1e9, unit="GB/s", cores=cpu_threads(),
+                            kind="oracle", seconds=dt, host_cpus=os.cpu_count(),
+                            sample=f"float64 numpy oracle, sequence 0, query heads 0..{heads - 1} "
+                                   f"of {cfg.n_q_heads} ({heads / cfg.n_q_heads / cfg.batch:.4f} "
+                                   f"of one step), {dt:.2f} s")
+
+    if rank == 0:
+        n_tok = sum(seq_lens)
+        line = dict(
+            metric=METRIC, value=head["gbs"], unit="GB/s", n_gpus=world, steps=args.steps,
+            warmup=args.warmup, ms_per_step=head["ms"], higher_is_better=True, scaling="weak",
+            vs_baseline=None, dtype="f32", data="synthetic",
+            config=dict(workload=cfg.name, batch=cfg.batch, context=cfg.max_seq_len,
+                        n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads, head_dim=cfg.head_dim,
+                        kv_dtype=cfg.dtype, page_size=cfg.page_size, n_list=cfg.n_list,
+                        pq_m=cfg.pq_m, budget_ppm=cfg.budget_ppm, kmeans_iters=cfg.kmeans_iters,
+                        l2="flushed between steps by a 512 MiB device write (not timed); "
+                           "per-step CUDA events on the launch stream",
+                        input_generation_s=round(t_gen, 1)),
+            us_per_step=1000 * head["ms"], us_p10=1000 * head["p10"], us_p50=1000 * head["p50"],
+            us_p90=1000 * head["p90"],
+            pct_of_8TBps=100 * head["gbs"] / world / NOMINAL_HBM_GBS,
+            pct_of_measured_peak=100 * head["gbs"] / world / peak,
+            decode_tokens_per_s=world * cfg.batch / (head["ms"] * 1e-3),
+            key_tokens_scanned_per_s=world * cfg.n_kv_heads * n_tok / (head["ms"] * 1e-3),
+            algorithmic_bytes_per_step=head["bytes"], dense_attention_bytes=dense_attention_bytes(cfg, seq_lens),
+            clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
+            cpu_baseline=cpu_baseline, variants=variants,
+            context_only="paper: 1.58x over FlashAttention-3 on one H20 at 128K, 1% (other "
+                         "hardware, other index setting)")
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -157,6 +157,15 @@ int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* i
                  const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out,
                  void* ws, size_t ws_bytes, void* stream);
 
+/* pqhsa_decode that also records five caller-created CUDA events (cudaEvent_t passed as
+ * void*, in a HOST array) on `stream`: [0] before the first launch, [1] before the scan,
+ * [2] before the top-k, [3] before the hybrid attention, [4] after the last kernel.  For
+ * per-stage timing; the kernels and their launch configuration are those of pqhsa_decode. */
+#define PQHSA_N_STAGE_EVENTS 5
+int pqhsa_decode_events(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                        const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out,
+                        void* ws, size_t ws_bytes, void* stream, void* const* stage_events);
+
 /* pqhsa_decode for a caller whose query and output live in HOST memory (pinned for the
  * copies to be asynchronous): copies q_host -> q_dev_staging, runs the step, copies
  * out_dev_staging -> out_host and waits for the stream.  The index, the KV cache and

@@ -72,19 +72,21 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.upb = o.Hkv * o.n_hg;
   o.n_part = o.scan_ctas / o.upb + 2;
   o.rows = o.B * o.Hq;
-  if (scan_smem_bytes(o, true) <= kMaxSmemPerCta) o.coarse_in_smem = 1;
+  // the coarse table is bulk-copied: its byte size and unit stride must be multiples of 16
+  if (scan_smem_bytes(o, true) <= kMaxSmemPerCta && (o.Gc * o.n_list) % 4 == 0) o.coarse_in_smem = 1;
   else if (scan_smem_bytes(o, false) <= kMaxSmemPerCta) o.coarse_in_smem = 0;
   else return PQHSA_ERR_UNSUPPORTED;
 
-  o.hist_chunks = ceil_div(2LL * o.num_sms, o.rows);
-  const int max_chunks = o.N_max / 4096 > 0 ? o.N_max / 4096 : 1;
-  if (o.hist_chunks > max_chunks) o.hist_chunks = max_chunks;
-  if (o.hist_chunks < 1) o.hist_chunks = 1;
+  o.hist_chunks = ceil_div(o.N_max, kSelChunk);
   o.cand_cap = o.N_max / 4 > 4096 ? o.N_max / 4 : 4096;
   if (o.cand_cap > o.N_max) o.cand_cap = o.N_max;
-  o.splits = ceil_div(4LL * o.num_sms, o.rows);
-  const int max_splits = (o.k_max + o.n_list / 4) / 32 > 0 ? (o.k_max + o.n_list / 4) / 32 : 1;
-  if (o.splits > max_splits) o.splits = max_splits;
+  // split-K CTAs per row: about 96 selected tokens each, but enough CTAs to fill the GPU
+  // when there are few rows, as long as every CTA keeps at least 32 units of work
+  o.splits = ceil_div(o.k_max, 96);
+  int fill = ceil_div(4LL * o.num_sms, o.rows);
+  const int max_fill = (o.k_max + o.n_list / 4) / 32 > 0 ? (o.k_max + o.n_list / 4) / 32 : 1;
+  if (fill > max_fill) fill = max_fill;
+  if (o.splits < fill) o.splits = fill;
   if (o.splits > 64) o.splits = 64;
   if (o.splits < 1) o.splits = 1;
   return PQHSA_OK;
@@ -217,7 +219,7 @@ int pqhsa_decode_launch_count(const pqhsa_params* params) {
   Plan pl;
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
-  return 7;   // memset, LUT build, scan, select histogram, select filter, background prep, attend
+  return 6;   // LUT build, scan, select histogram, select filter, background prep, attend
 }
 
 int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index* index,
@@ -228,7 +230,8 @@ int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index
   if ((rc = check_index(index)) != PQHSA_OK) return rc;
   if (q == nullptr || lut == nullptr || coarse == nullptr || !aligned16(lut) || !aligned16(coarse))
     return PQHSA_ERR_INVALID_ARG;
-  return cuda_status(launch_build_lut(pl, q, *index, lut, coarse, static_cast<cudaStream_t>(stream)));
+  return cuda_status(launch_build_lut(pl, q, *index, lut, coarse, nullptr, 0,
+                                      static_cast<cudaStream_t>(stream)));
 }
 
 int pqhsa_scan(const pqhsa_params* params, const pqhsa_index* index, const float* lut,
@@ -291,9 +294,9 @@ int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_p
                                    sel_count, seq_lens, out, lse_or_null, st));
 }
 
-int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* index,
-                 const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out, void* ws,
-                 size_t ws_bytes, void* stream) {
+static int decode_impl(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                       const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out, void* ws,
+                       size_t ws_bytes, void* stream, void* const* ev) {
   Plan pl;
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
@@ -312,16 +315,40 @@ int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* i
   int32_t* sel_idx = reinterpret_cast<int32_t*>(w + L.sel_idx);
   int32_t* sel_count = reinterpret_cast<int32_t*>(w + L.sel_count);
   float* kth = reinterpret_cast<float*>(w + L.kth);
-  if (cudaMemsetAsync(w + L.zero_begin, 0, L.zero_bytes, st) != cudaSuccess) return PQHSA_ERR_CUDA;
-  cudaError_t e = launch_build_lut(pl, q, *index, lut, coarse, st);
+  auto mark = [&](int i) {
+    return ev == nullptr ? cudaSuccess : cudaEventRecord(static_cast<cudaEvent_t>(ev[i]), st);
+  };
+  cudaError_t e = mark(0);
+  // the LUT kernel also clears the status word, histograms, counters and tickets
+  if (e == cudaSuccess)
+    e = launch_build_lut(pl, q, *index, lut, coarse, w + L.zero_begin, L.zero_bytes, st);
+  if (e == cudaSuccess) e = mark(1);
   if (e == cudaSuccess)
     e = launch_scan(pl, *index, lut, coarse, seq_lens, scores, partials,
                     reinterpret_cast<int*>(w + L.status), st);
+  if (e == cudaSuccess) e = mark(2);
   if (e == cudaSuccess) e = launch_select(pl, L, w, scores, seq_lens, sel_idx, sel_count, kth, st);
+  if (e == cudaSuccess) e = mark(3);
   if (e == cudaSuccess)
     e = launch_attend(pl, L, w, q, *kv, *index, scores, partials, sel_idx, sel_count, seq_lens,
                       out, nullptr, st);
+  if (e == cudaSuccess) e = mark(4);
   return cuda_status(e);
+}
+
+int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                 const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out, void* ws,
+                 size_t ws_bytes, void* stream) {
+  return decode_impl(params, q, index, kv, seq_lens, out, ws, ws_bytes, stream, nullptr);
+}
+
+int pqhsa_decode_events(const pqhsa_params* params, const void* q, const pqhsa_index* index,
+                        const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out, void* ws,
+                        size_t ws_bytes, void* stream, void* const* stage_events) {
+  if (stage_events == nullptr) return PQHSA_ERR_INVALID_ARG;
+  for (int i = 0; i < PQHSA_N_STAGE_EVENTS; ++i)
+    if (stage_events[i] == nullptr) return PQHSA_ERR_INVALID_ARG;
+  return decode_impl(params, q, index, kv, seq_lens, out, ws, ws_bytes, stream, stage_events);
 }
 
 int pqhsa_decode_host(const pqhsa_params* params, const void* q_host, void* q_dev_staging,

@@ -16,7 +16,7 @@ namespace pqhsa {
 
 namespace {
 
-constexpr int kBgThreads = 256;
+constexpr int kBgThreads = 512;
 constexpr int kPartStride = 2 + kHeadDim;     // m, Z, N[128]
 
 __global__ void __launch_bounds__(kBgThreads)
@@ -24,8 +24,9 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
                const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_count,
                const uint16_t* __restrict__ lids, const int32_t* __restrict__ seq_lens,
                float* __restrict__ bg_mass, float* __restrict__ bg_max) {
-  extern __shared__ float s_tot[];            // [n_list]
-  __shared__ float s_m;
+  extern __shared__ float s_dyn[];            // [n_list] sums, then [n_part] segment scales
+  float* s_tot = s_dyn;
+  float* s_scale = s_dyn + pl.n_list;
   const int row = blockIdx.x, tid = threadIdx.x;
   const int b = row / pl.Hq, h = row % pl.Hq;
   const int kv = h / pl.G, hg = (h % pl.G) / pl.Gc;
@@ -37,6 +38,12 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
     if (tid == 0) bg_max[row] = -CUDART_INF_F;
     return;
   }
+  // the selected tokens' scores and list ids: issue these gathers first
+  const int cnt = sel_count[row];
+  const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
+  const float* rs = scores + (size_t)row * pl.N_max;
+  const uint16_t* rl = lids + ((size_t)b * pl.Hkv + kv) * pl.N_max;
+
   // which scan segments cover this row's unit
   const ScanSplit sp = scan_split(seq_lens, pl.B, pl.N_max, pl.upb, pl.scan_ctas);
   long long base = 0;
@@ -47,36 +54,54 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   const int nseg = split_cta_of(sp, s_u + tb - 1) - c_first + 1;
   const float* pr = partials + (size_t)row * pl.n_part * (n_list + 1);
 
-  if (tid == 0) {
-    float m = -CUDART_INF_F;
-    for (int s = 0; s < nseg; ++s) m = fmaxf(m, pr[(size_t)s * (n_list + 1)]);
-    s_m = m;
-  }
+  if (tid < nseg) s_scale[tid] = pr[(size_t)tid * (n_list + 1)];     // segment maxima
   __syncthreads();
-  const float m2 = s_m * kLog2e;
+  float m = -CUDART_INF_F;
+  for (int s = 0; s < nseg; ++s) m = fmaxf(m, s_scale[s]);
+  const float m2 = m * kLog2e;
+  __syncthreads();
+  if (tid < nseg) s_scale[tid] = fast_exp2(fmaf(s_scale[tid], kLog2e, -m2));
+  __syncthreads();
   for (int j = tid; j < n_list; j += kBgThreads) {
     float acc = 0.f;
-    for (int s = 0; s < nseg; ++s) {
-      const float* ps = pr + (size_t)s * (n_list + 1);
-      const float v = ps[1 + j];
-      if (v != 0.f) acc = fmaf(v, fast_exp2(fmaf(ps[0], kLog2e, -m2)), acc);
+    int s = 0;
+    for (; s + 4 <= nseg; s += 4) {
+      float v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = pr[(size_t)(s + u) * (n_list + 1) + 1 + j];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) acc = fmaf(v[u], s_scale[s + u], acc);
     }
+    for (; s < nseg; ++s) acc = fmaf(pr[(size_t)s * (n_list + 1) + 1 + j], s_scale[s], acc);
     s_tot[j] = acc;
   }
   __syncthreads();
   // take the selected tokens out of their lists' sums
-  const int cnt = sel_count[row];
-  const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
-  const float* rs = scores + (size_t)row * pl.N_max;
-  const uint16_t* rl = lids + ((size_t)b * pl.Hkv + kv) * pl.N_max;
-  for (int t = tid; t < cnt; t += kBgThreads) {
-    const int i = sel[t];
-    const float x = fmaf(rs[i], kLog2e, -m2);
-    if (x > kNegligibleLog2) atomicAdd(&s_tot[rl[i]], -fast_exp2(x));
+  for (int t0 = 0; t0 < cnt; t0 += kBgThreads * 2) {
+    int idx[2];
+    float sc[2];
+    uint32_t li[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int t = t0 + u * kBgThreads + tid;
+      idx[u] = t < cnt ? sel[t] : -1;
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      sc[u] = idx[u] >= 0 ? rs[idx[u]] : 0.f;
+      li[u] = idx[u] >= 0 ? rl[idx[u]] : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (idx[u] >= 0) {
+        const float x = fmaf(sc[u], kLog2e, -m2);
+        if (x > kNegligibleLog2) atomicAdd(&s_tot[li[u]], -fast_exp2(x));
+      }
+    }
   }
   __syncthreads();
   for (int j = tid; j < n_list; j += kBgThreads) mass[j] = fmaxf(s_tot[j], 0.f);
-  if (tid == 0) bg_max[row] = s_m;
+  if (tid == 0) bg_max[row] = m;
 }
 
 template <typename T> struct Unpack;
@@ -118,7 +143,7 @@ __device__ __forceinline__ float safe_scale(float m_from, float m_to, float Z) {
 }
 
 template <typename T, int U>
-__global__ void __launch_bounds__(kAttendThreads)
+__global__ void __launch_bounds__(kAttendThreads, 4)
 attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
               long long stride_page, long long stride_token, long long stride_head,
               const int32_t* __restrict__ block_table, const int32_t* __restrict__ sel_idx,
@@ -137,30 +162,61 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   const size_t ukv = (size_t)b * pl.Hkv + kv;
   const int n_list = pl.n_list;
   const int cnt = sel_count[row];
+
+  // ---- this warp's slice of the selected tokens: resolve cache offsets first (two
+  //      dependent loads: position, then page id), so they overlap the background part
+  const int tl = (int)((long long)split * cnt / S);
+  const int th = (int)((long long)(split + 1) * cnt / S);
+  const int per_warp = (th - tl + kWarps - 1) / kWarps;
+  const int wl = min(th, tl + warp * per_warp), wh = min(th, wl + per_warp);
+  const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
+  const int32_t* bt = block_table + (size_t)b * pl.max_pages;
+  int my_pos = (wl + lane < wh) ? sel[wl + lane] : -1;
+
   const float m_bg = bg_max[row] * kLog2e;    // reference of the background masses (log2 units)
 
   // ---- background slice: Z += M_j, N += M_j * vbar_j  (all relative to m_bg)
   {
     const int jl = (int)((long long)split * n_list / S);
     const int jh = (int)((long long)(split + 1) * n_list / S);
+    const int per = (jh - jl + kWarps - 1) / kWarps;
+    const int a = min(jh, jl + warp * per), e = min(jh, a + per);
     const float* mass = bg_mass + (size_t)row * n_list;
+    const float4* vm = reinterpret_cast<const float4*>(vmeans + ukv * n_list * kHeadDim);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
-    for (int j = jl + warp; j < jh; j += kWarps) {
-      const float mj = mass[j];
-      if (mj > 0.f) {
-        const float4 v = __ldg(reinterpret_cast<const float4*>(
-                                   vmeans + (ukv * n_list + j) * kHeadDim) + lane);
-        acc.x = fmaf(mj, v.x, acc.x); acc.y = fmaf(mj, v.y, acc.y);
-        acc.z = fmaf(mj, v.z, acc.z); acc.w = fmaf(mj, v.w, acc.w);
-        z += mj;
+    for (int j0 = a; j0 < e; j0 += 32) {
+      const float mine = (j0 + lane < e) ? mass[j0 + lane] : 0.f;
+      unsigned live = __ballot_sync(0xffffffffu, mine > 0.f);
+      while (live) {
+        int jj[4];
+        float mj[4];
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          jj[u] = live ? __ffs(live) - 1 : -1;
+          if (live) live &= live - 1;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          mj[u] = __shfl_sync(0xffffffffu, mine, jj[u] < 0 ? 0 : jj[u]);
+          v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (jj[u] >= 0) v[u] = __ldg(vm + (size_t)(j0 + jj[u]) * (kHeadDim / 4) + lane);
+          else mj[u] = 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          acc.x = fmaf(mj[u], v[u].x, acc.x); acc.y = fmaf(mj[u], v[u].y, acc.y);
+          acc.z = fmaf(mj[u], v[u].z, acc.z); acc.w = fmaf(mj[u], v[u].w, acc.w);
+          z += mj[u];
+        }
       }
     }
     *reinterpret_cast<float4*>(&s_N[kWarps + warp][4 * lane]) = acc;
     if (lane == 0) { s_m[kWarps + warp] = m_bg; s_Z[kWarps + warp] = z; }
   }
 
-  // ---- exact slice: selected tokens [tl, th) of this row
+  // ---- exact slice
   const int gi = lane >> 3, gl = lane & 7;      // lane group (4 per warp) and lane in group
   float qf[16];
   {
@@ -178,20 +234,15 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
 #pragma unroll
   for (int t = 0; t < 16; ++t) st.acc[t] = 0.f;
 
-  const int tl = (int)((long long)split * cnt / S);
-  const int th = (int)((long long)(split + 1) * cnt / S);
-  const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
-  const int32_t* bt = block_table + (size_t)b * pl.max_pages;
-  for (int base = tl + warp * 32; base < th; base += kWarps * 32) {
-    // each lane resolves the cache offset of one token of the batch
+  for (int base = wl; base < wh; base += 32) {
+    if (base != wl) my_pos = (base + lane < wh) ? sel[base + lane] : -1;
     long long off = 0;
-    if (base + lane < th) {
-      const int pos = sel[base + lane];
-      const int page = __ldg(bt + pos / pl.page_size);
-      off = (long long)page * stride_page + (long long)(pos % pl.page_size) * stride_token +
+    if (my_pos >= 0) {
+      const int page = __ldg(bt + my_pos / pl.page_size);
+      off = (long long)page * stride_page + (long long)(my_pos % pl.page_size) * stride_token +
             (long long)kv * stride_head;
     }
-    const int nb = min(32, th - base);
+    const int nb = min(32, wh - base);
     for (int j0 = 0; j0 < nb; j0 += 4 * U) {
       uint4 kr[U][2], vr[U][2];
       bool ok[U];
@@ -295,11 +346,21 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   for (int s = 0; s < S; ++s)
     if (__ldcg(pr + s * kPartStride + 1) > 0.f) m_r = fmaxf(m_r, __ldcg(pr + s * kPartStride));
   float Z_r = 0.f, N_r = 0.f;
-  for (int s = 0; s < S; ++s) {
-    const float Zs = __ldcg(pr + s * kPartStride + 1);
-    const float a = safe_scale(__ldcg(pr + s * kPartStride), m_r, Zs);
-    Z_r = fmaf(Zs, a, Z_r);
-    N_r = fmaf(__ldcg(pr + s * kPartStride + 2 + tid), a, N_r);
+  for (int s0 = 0; s0 < S; s0 += 4) {
+    float Zs[4], ms[4], Ns[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int s = s0 + u;
+      Zs[u] = s < S ? __ldcg(pr + s * kPartStride + 1) : 0.f;
+      ms[u] = s < S ? __ldcg(pr + s * kPartStride) : 0.f;
+      Ns[u] = s < S ? __ldcg(pr + s * kPartStride + 2 + tid) : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float a = safe_scale(ms[u], m_r, Zs[u]);
+      Z_r = fmaf(Zs[u], a, Z_r);
+      N_r = fmaf(Ns[u], a, N_r);
+    }
   }
   out[(size_t)row * kHeadDim + tid] = Unpack<T>::pack(Z_r > 0.f ? N_r / Z_r : 0.f);
   if (lse != nullptr && tid == 0)
@@ -317,19 +378,19 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
   float* bg_max = reinterpret_cast<float*>(ws + L.bg_max);
   float* split_part = reinterpret_cast<float*>(ws + L.split_part);
   uint32_t* tickets = reinterpret_cast<uint32_t*>(ws + L.attend_tickets);
-  bg_prep_kernel<<<pl.rows, kBgThreads, pl.n_list * sizeof(float), st>>>(
+  bg_prep_kernel<<<pl.rows, kBgThreads, (pl.n_list + pl.n_part) * sizeof(float), st>>>(
       pl, scores, list_partials, sel_idx, sel_count, ix.list_ids, seq_lens, bg_mass, bg_max);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 grid(pl.splits, pl.rows);
   if (pl.dtype == PQHSA_F16)
-    attend_kernel<__half, 2><<<grid, kAttendThreads, 0, st>>>(
+    attend_kernel<__half, 4><<<grid, kAttendThreads, 0, st>>>(
         pl, static_cast<const __half*>(q), static_cast<const __half*>(kv.k_cache),
         static_cast<const __half*>(kv.v_cache), kv.stride_page, kv.stride_token, kv.stride_head,
         kv.block_table, sel_idx, sel_count, bg_mass, bg_max, ix.list_vmeans, split_part, tickets,
         static_cast<__half*>(out), lse);
   else
-    attend_kernel<__nv_bfloat16, 2><<<grid, kAttendThreads, 0, st>>>(
+    attend_kernel<__nv_bfloat16, 4><<<grid, kAttendThreads, 0, st>>>(
         pl, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kv.k_cache),
         static_cast<const __nv_bfloat16*>(kv.v_cache), kv.stride_page, kv.stride_token,
         kv.stride_head, kv.block_table, sel_idx, sel_count, bg_mass, bg_max, ix.list_vmeans,

@@ -18,6 +18,7 @@ constexpr int kScanThreads = 512;
 constexpr int kScanMinTiles = kScanThreads / 32;   // a scan CTA gets at least one tile per warp
 constexpr int kHistBins = 4096;      // 12-bit radix digits for the two coarse select levels
 constexpr int kSelThreads = 512;
+constexpr int kSelChunk = 8192;      // scores per select CTA: 16 per thread, kept in registers
 constexpr int kAttendThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegligibleLog2 = -64.0f;   // exp2 arguments below this add nothing to a sum
@@ -35,7 +36,7 @@ struct Plan {
   int n_part;                        // list-partial slots per score row
   int upb;                           // scan units per sequence = Hkv * n_hg
   int rows;                          // B * Hq score rows
-  int hist_chunks;                   // CTAs per row in the select kernels
+  int hist_chunks;                   // CTAs per row in the select kernels: ceil(N_max / kSelChunk)
   int cand_cap;                      // candidate slots per row
   int splits;                        // split-K CTAs per row in the attend kernel
   int coarse_in_smem;                // scan keeps the coarse table in shared memory
@@ -134,8 +135,9 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // ------------------------------------------------------------------ stage launchers
 // Each returns a cudaError_t from the launch (cudaSuccess if nothing had to run).
+// zero_ptr / zero_bytes: optional region (16-byte granules) the kernel clears on the side.
 cudaError_t launch_build_lut(const Plan& pl, const void* q, const pqhsa_index& ix, float* lut,
-                             float* coarse, cudaStream_t st);
+                             float* coarse, void* zero_ptr, size_t zero_bytes, cudaStream_t st);
 cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,
                         const float* coarse, const int32_t* seq_lens, float* scores,
                         float* list_partials, int* status, cudaStream_t st);

@@ -2,21 +2,24 @@
 // T(q) = TopK_{k, i in R} l~_i with k = ceil(rho |R|).
 //
 // Radix threshold select on order-preserving 32-bit keys, digits of 12 / 12 / 8 bits:
-//   hist kernel    every CTA histograms the top digit of its chunk of a row; the last CTA of
-//                  the row to finish finds the digit b1 that holds the k-th largest key;
-//   filter kernel  keys above b1 are winners and are emitted at once; keys inside b1 are
-//                  appended to a candidate list and histogrammed on the second digit; the
-//                  last CTA of the row resolves the remaining two digits on the candidates.
-// Equal keys at the threshold are taken in order of position (lowest first), which is the
-// stable rule of a full sort.  No CTA ever waits for another: "last CTA" is decided by an
-// atomic ticket.
+//   hist kernel    every CTA histograms the top digit of its 8192-score chunk of a row; the
+//                  last CTA of the row to finish finds the digit b1 that holds the k-th key;
+//   filter kernel  keys above b1 are winners and are written out at once; keys inside b1
+//                  are appended to a candidate list and histogrammed on the second digit;
+//                  the last CTA of the row resolves the remaining two digits on the
+//                  candidates.
+// A CTA keeps its 16 scores per thread in registers, counts, takes its output slots with one
+// atomic per list, and writes.  Equal keys at the threshold are taken in order of position
+// (lowest first), the stable rule of a full sort.  No CTA ever waits for another: "last CTA"
+// is decided by an atomic ticket.
 #include "common.cuh"
 
 namespace pqhsa {
 
 namespace {
 
-struct RowState { int b1, k1, k, n; };
+constexpr int kElems = kSelChunk / kSelThreads;   // scores per thread (16)
+constexpr int kStashCap = 2048;
 
 // Largest digit D with  count(digits > D) < k <= count(digits >= D).  `hist` may be global
 // (read through L2) or shared.  All kSelThreads threads must call; k >= 1 and the histogram
@@ -28,12 +31,15 @@ __device__ void find_digit(const uint32_t* hist, int nbins, int k, int* s_scan, 
   const int per = (nbins + kSelThreads - 1) / kSelThreads;
   // thread t owns digits [hi - per, hi) with hi = nbins - t*per, walked from the top down
   const int hi = nbins - tid * per;
+  uint32_t mine[8];
   uint32_t local = 0;
-  for (int j = 0; j < per; ++j) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
     const int d = hi - 1 - j;
-    if (d >= 0) local += kGlobal ? __ldcg(hist + d) : hist[d];
+    mine[j] = (j < per && d >= 0) ? (kGlobal ? __ldcg(hist + d) : hist[d]) : 0u;
+    local += mine[j];
   }
-  // inclusive scan over threads (thread 0 = top digits)
+  if (tid == 0) { s_scan[32] = 0; s_scan[33] = 0; }
   uint32_t inc = local;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -54,19 +60,15 @@ __device__ void find_digit(const uint32_t* hist, int nbins, int k, int* s_scan, 
   }
   __syncthreads();
   const uint32_t before = (uint32_t)s_scan[warp] + inc - local;   // items in digits above mine
-  __syncthreads();
   if (before < (uint32_t)k && (uint32_t)k <= before + local) {
     uint32_t run = before;
-    for (int j = 0; j < per; ++j) {
-      const int d = hi - 1 - j;
-      if (d < 0) break;
-      const uint32_t c = kGlobal ? __ldcg(hist + d) : hist[d];
-      if (run + c >= (uint32_t)k) {
-        s_scan[32] = d;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (run < (uint32_t)k && run + mine[j] >= (uint32_t)k) {
+        s_scan[32] = hi - 1 - j;
         s_scan[33] = (int)run;
-        break;
       }
-      run += c;
+      run += mine[j];
     }
   }
   __syncthreads();
@@ -75,7 +77,8 @@ __device__ void find_digit(const uint32_t* hist, int nbins, int k, int* s_scan, 
   __syncthreads();
 }
 
-// Appends `flag`ged lanes' values through one atomic per warp; returns the slot or -1.
+// Slot for each `flag`ged lane through one atomic per warp (counter in shared or global
+// memory); -1 for the others.  All 32 lanes must call.
 __device__ __forceinline__ int warp_append(bool flag, uint32_t* counter) {
   const unsigned m = __ballot_sync(0xffffffffu, flag);
   if (m == 0) return -1;
@@ -87,11 +90,22 @@ __device__ __forceinline__ int warp_append(bool flag, uint32_t* counter) {
   return flag ? (int)(base + __popc(m & ((1u << lane) - 1u))) : -1;
 }
 
-__device__ __forceinline__ void row_chunk(int n, int chunks, int c, int& lo, int& hi) {
-  int per = (n + chunks - 1) / chunks;
-  per = (per + 3) & ~3;                      // keep float4 loads aligned
-  lo = min(n, c * per);
-  hi = min(n, lo + per);
+// The 16 scores of this thread: 4 float4 at float4-index chunk*2048 + j*512 + tid.
+__device__ __forceinline__ void load_chunk(const float* __restrict__ rs, int chunk, int n,
+                                           float (&v)[kElems], int (&pos0)[4]) {
+  const int tid = threadIdx.x;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int i = chunk * kSelChunk + (j * kSelThreads + tid) * 4;
+    pos0[j] = i;
+    if (i + 3 < n) {
+      const float4 f = __ldcg(reinterpret_cast<const float4*>(rs + i));
+      v[4 * j] = f.x; v[4 * j + 1] = f.y; v[4 * j + 2] = f.z; v[4 * j + 3] = f.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[4 * j + e] = (i + e < n) ? __ldcg(rs + i + e) : 0.f;
+    }
+  }
 }
 
 // ------------------------------------------------------------------------- hist kernel
@@ -103,12 +117,12 @@ sel_hist_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __rest
   __shared__ uint32_t s_hist[kHistBins];
   __shared__ int s_scan[34];
   __shared__ int s_last;
-  const int row = blockIdx.y, tid = threadIdx.x;
+  const int row = blockIdx.y, tid = threadIdx.x, chunk = blockIdx.x;
   const int b = row / pl.Hq;
   const int n = clamp_len(seq_lens[b], pl.N_max);
   const int k = budget_k(n, pl.ppm);
   if (k == 0) {
-    if (blockIdx.x == 0 && tid == 0) {
+    if (chunk == 0 && tid == 0) {
       rowstate[row * 4 + 0] = -1; rowstate[row * 4 + 1] = 0;
       rowstate[row * 4 + 2] = 0;  rowstate[row * 4 + 3] = n;
       sel_count[row] = 0;
@@ -116,27 +130,21 @@ sel_hist_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __rest
     }
     return;
   }
-  for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
-  __syncthreads();
-  int lo, hi;
-  row_chunk(n, gridDim.x, blockIdx.x, lo, hi);
-  const float* rs = scores + (size_t)row * pl.N_max;
-  for (int i = lo + tid * 4; i < hi; i += kSelThreads * 4) {
-    if (i + 3 < hi) {
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(rs + i));
-      atomicAdd(&s_hist[score_key(v.x) >> 20], 1u);
-      atomicAdd(&s_hist[score_key(v.y) >> 20], 1u);
-      atomicAdd(&s_hist[score_key(v.z) >> 20], 1u);
-      atomicAdd(&s_hist[score_key(v.w) >> 20], 1u);
-    } else {
-      for (int j = i; j < hi; ++j) atomicAdd(&s_hist[score_key(__ldcg(rs + j)) >> 20], 1u);
-    }
-  }
-  __syncthreads();
   uint32_t* gh = hist1 + (size_t)row * kHistBins;
-  for (int i = tid; i < kHistBins; i += kSelThreads)
-    if (s_hist[i]) atomicAdd(gh + i, s_hist[i]);
-  __threadfence();
+  if (chunk * kSelChunk < n) {
+    float v[kElems];
+    int pos0[4];
+    load_chunk(scores + (size_t)row * pl.N_max, chunk, n, v, pos0);
+    for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < kElems; ++e)
+      if (pos0[e >> 2] + (e & 3) < n) atomicAdd(&s_hist[score_key(v[e]) >> 20], 1u);
+    __syncthreads();
+    for (int i = tid; i < kHistBins; i += kSelThreads)
+      if (s_hist[i]) atomicAdd(gh + i, s_hist[i]);
+    __threadfence();
+  }
   __syncthreads();
   if (tid == 0) s_last = (atomicAdd(&counters[row * 4 + 0], 1u) == gridDim.x - 1);
   __syncthreads();
@@ -159,22 +167,36 @@ template <class F>
 __device__ __forceinline__ void for_each_candidate(bool overflow, const uint2* cand, int n_stored,
                                                    const float* rs, int n, uint32_t b1, F f) {
   const int tid = threadIdx.x;
+  constexpr int U = 4;
   if (!overflow) {
-    for (int base = 0; base < n_stored; base += kSelThreads) {
-      const int i = base + tid;
-      const bool v = i < n_stored;
-      uint2 c = make_uint2(0u, 0u);
-      if (v) c = __ldcg(cand + i);
-      f(v, c.x, (int)c.y);
+    for (int base = 0; base < n_stored; base += kSelThreads * U) {
+      uint2 c[U];
+      bool v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = base + u * kSelThreads + tid;
+        v[u] = i < n_stored;
+        c[u] = make_uint2(0u, 0u);
+        if (v[u]) c[u] = __ldcg(cand + i);
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) f(v[u], c[u].x, (int)c[u].y);
     }
   } else {
-    for (int base = 0; base < n; base += kSelThreads) {
-      const int i = base + tid;
-      bool v = i < n;
-      uint32_t key = 0u;
-      if (v) key = score_key(__ldcg(rs + i));
-      v = v && (key >> 20) == b1;
-      f(v, key, i);
+    for (int base = 0; base < n; base += kSelThreads * U) {
+      float s[U];
+      bool v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = base + u * kSelThreads + tid;
+        v[u] = i < n;
+        s[u] = v[u] ? __ldcg(rs + i) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint32_t key = score_key(s[u]);
+        f(v[u] && (key >> 20) == b1, key, base + u * kSelThreads + tid);
+      }
     }
   }
 }
@@ -200,49 +222,85 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, const uint32_t* __r
                   int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_count,
                   float* __restrict__ kth, int* __restrict__ status) {
   __shared__ uint32_t s_hist[kHistBins];
+  __shared__ uint2 s_stash[kStashCap];
   __shared__ int s_scan[34];
   __shared__ int s_last;
-  const int row = blockIdx.y, tid = threadIdx.x;
+  __shared__ uint32_t s_base[2], s_cnt[2];
+  const int row = blockIdx.y, tid = threadIdx.x, chunk = blockIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
   const int b1 = rowstate[row * 4 + 0], k1 = rowstate[row * 4 + 1];
   const int k = rowstate[row * 4 + 2], n = rowstate[row * 4 + 3];
   if (k == 0) return;
-  for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
-  __syncthreads();
-  int lo, hi;
-  row_chunk(n, gridDim.x, blockIdx.x, lo, hi);
   const float* rs = scores + (size_t)row * pl.N_max;
   int32_t* out = sel_idx + (size_t)row * pl.k_max;
   uint2* rc = cand + (size_t)row * pl.cand_cap;
   uint32_t* n_out = &counters[row * 4 + 2];
   uint32_t* n_cand = &counters[row * 4 + 3];
-
-  for (int base = lo; base < hi; base += kSelThreads * 4) {
-    const int i = base + tid * 4;
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
-    if (i + 3 < hi) {
-      const float4 f4 = __ldcg(reinterpret_cast<const float4*>(rs + i));
-      v[0] = f4.x; v[1] = f4.y; v[2] = f4.z; v[3] = f4.w;
-    } else {
-      for (int j = 0; j < 4; ++j) if (i + j < hi) v[j] = __ldcg(rs + i + j);
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const bool valid = i + j < hi;
-      const uint32_t key = score_key(v[j]);
-      const int bin = (int)(key >> 20);
-      const int p = warp_append(valid && bin > b1, n_out);
-      if (p >= 0 && p < pl.k_max) out[p] = i + j;
-      const bool is_c = valid && bin == b1;
-      if (is_c) atomicAdd(&s_hist[(key >> 8) & 0xfffu], 1u);
-      const int pc = warp_append(is_c, n_cand);
-      if (pc >= 0 && pc < pl.cand_cap) rc[pc] = make_uint2(key, (uint32_t)(i + j));
-    }
-  }
-  __syncthreads();
   uint32_t* gh = hist2 + (size_t)row * kHistBins;
-  for (int i = tid; i < kHistBins; i += kSelThreads)
-    if (s_hist[i]) atomicAdd(gh + i, s_hist[i]);
-  __threadfence();
+
+  if (chunk * kSelChunk < n) {
+    float v[kElems];
+    int pos0[4];
+    load_chunk(rs, chunk, n, v, pos0);
+    for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
+    __syncthreads();
+    uint32_t keys[kElems];
+    uint32_t win_mask = 0, cand_mask = 0;
+#pragma unroll
+    for (int e = 0; e < kElems; ++e) {
+      keys[e] = score_key(v[e]);
+      const bool valid = pos0[e >> 2] + (e & 3) < n;
+      const int bin = (int)(keys[e] >> 20);
+      if (valid && bin > b1) win_mask |= 1u << e;
+      if (valid && bin == b1) {
+        cand_mask |= 1u << e;
+        atomicAdd(&s_hist[(keys[e] >> 8) & 0xfffu], 1u);
+      }
+    }
+    // exclusive scan of (winners << 16 | candidates) over the CTA
+    const uint32_t mine = ((uint32_t)__popc(win_mask) << 16) | (uint32_t)__popc(cand_mask);
+    uint32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += u;
+    }
+    if (lane == 31) s_scan[warp] = (int)inc;
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t wv = (lane < kSelThreads / 32) ? (uint32_t)s_scan[lane] : 0u;
+      uint32_t ws = wv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t u = __shfl_up_sync(0xffffffffu, ws, o);
+        if (lane >= o) ws += u;
+      }
+      if (lane < kSelThreads / 32) s_scan[lane] = (int)(ws - wv);
+      if (lane == kSelThreads / 32 - 1) {        // CTA totals: take the output slots
+        const uint32_t tw = ws >> 16, tc = ws & 0xffffu;
+        s_base[0] = tw ? atomicAdd(n_out, tw) : 0u;
+        s_base[1] = tc ? atomicAdd(n_cand, tc) : 0u;
+      }
+    }
+    __syncthreads();
+    const uint32_t excl = (uint32_t)s_scan[warp] + inc - mine;
+    uint32_t pw = s_base[0] + (excl >> 16), pc = s_base[1] + (excl & 0xffffu);
+#pragma unroll
+    for (int e = 0; e < kElems; ++e) {
+      const int pos = pos0[e >> 2] + (e & 3);
+      if (win_mask & (1u << e)) {
+        if (pw < (uint32_t)pl.k_max) out[pw] = pos;
+        ++pw;
+      }
+      if (cand_mask & (1u << e)) {
+        if (pc < (uint32_t)pl.cand_cap) rc[pc] = make_uint2(keys[e], (uint32_t)pos);
+        ++pc;
+      }
+    }
+    for (int i = tid; i < kHistBins; i += kSelThreads)
+      if (s_hist[i]) atomicAdd(gh + i, s_hist[i]);
+    __threadfence();
+  }
   __syncthreads();
   if (tid == 0) s_last = (atomicAdd(&counters[row * 4 + 1], 1u) == gridDim.x - 1);
   __syncthreads();
@@ -253,54 +311,81 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, const uint32_t* __r
   const int n_in_bin = (int)__ldcg(hist1 + (size_t)row * kHistBins + b1);
   const bool overflow = n_in_bin > pl.cand_cap;
   const int n_stored = overflow ? 0 : n_in_bin;
+  const uint32_t base_out = __ldcg(n_out);          // winners written by the main phase
   int b2, above2;
   find_digit<true>(gh, kHistBins, k1, s_scan, b2, above2);
   const int k2 = k1 - above2;
   for (int i = tid; i < 256; i += kSelThreads) s_hist[i] = 0u;
+  if (tid == 0) { s_cnt[0] = 0u; s_cnt[1] = 0u; }
   __syncthreads();
+  // one pass: second digit above b2 -> winner; equal -> third-digit histogram + stash
   for_each_candidate(overflow, rc, n_stored, rs, n, (uint32_t)b1,
                      [&](bool v, uint32_t key, int pos) {
                        const int d2 = (int)((key >> 8) & 0xfffu);
-                       const int p = warp_append(v && d2 > b2, n_out);
-                       if (p >= 0 && p < pl.k_max) out[p] = pos;
-                       if (v && d2 == b2) atomicAdd(&s_hist[key & 0xffu], 1u);
+                       const int p = warp_append(v && d2 > b2, &s_cnt[0]);
+                       if (p >= 0 && base_out + p < (uint32_t)pl.k_max) out[base_out + p] = pos;
+                       const bool tie = v && d2 == b2;
+                       if (tie) atomicAdd(&s_hist[key & 0xffu], 1u);
+                       const int ps = warp_append(tie, &s_cnt[1]);
+                       if (ps >= 0 && ps < kStashCap) s_stash[ps] = make_uint2(key, (uint32_t)pos);
                      });
   __syncthreads();
   int b3, above3;
   find_digit<false>(s_hist, 256, k2, s_scan, b3, above3);
   const int k3 = k2 - above3;                      // how many keys equal to the k-th are taken
   const int ties = (int)s_hist[b3];
+  const int n_stash = (int)s_cnt[1];
+  const bool stash_ok = n_stash <= kStashCap;
   const uint32_t kstar = ((uint32_t)b1 << 20) | ((uint32_t)b2 << 8) | (uint32_t)b3;
   int max_tie_pos = n;                             // take ties at positions <= this
   if (ties != k3) {
-    // k3-th smallest position among the ties, by bisection on the position
+    // k3-th smallest position among the keys equal to the k-th, by bisection on the position
     int plo = 0, phi = n - 1;
     while (plo < phi) {
       const int mid = plo + (phi - plo) / 2;
       int local = 0;
-      for_each_candidate(overflow, rc, n_stored, rs, n, (uint32_t)b1,
-                         [&](bool v, uint32_t key, int pos) {
-                           if (v && key == kstar && pos <= mid) ++local;
-                         });
+      if (stash_ok) {
+        for (int i = tid; i < n_stash; i += kSelThreads)
+          if (s_stash[i].x == kstar && (int)s_stash[i].y <= mid) ++local;
+      } else {
+        for_each_candidate(overflow, rc, n_stored, rs, n, (uint32_t)b1,
+                           [&](bool v, uint32_t key, int pos) {
+                             if (v && key == kstar && pos <= mid) ++local;
+                           });
+      }
       const int cnt = block_count(local, s_scan);
       if (cnt >= k3) phi = mid; else plo = mid + 1;
     }
     max_tie_pos = plo;
   }
-  for_each_candidate(overflow, rc, n_stored, rs, n, (uint32_t)b1,
-                     [&](bool v, uint32_t key, int pos) {
-                       const bool pre = v && (int)((key >> 8) & 0xfffu) == b2;
-                       const int low = (int)(key & 0xffu);
-                       const bool take = pre && (low > b3 || (low == b3 && pos <= max_tie_pos));
-                       const int p = warp_append(take, n_out);
-                       if (p >= 0 && p < pl.k_max) out[p] = pos;
-                     });
+  if (stash_ok) {
+    for (int base = 0; base < n_stash; base += kSelThreads) {
+      const int i = base + tid;
+      bool take = false;
+      int pos = 0;
+      if (i < n_stash) {
+        const int low = (int)(s_stash[i].x & 0xffu);
+        pos = (int)s_stash[i].y;
+        take = low > b3 || (low == b3 && pos <= max_tie_pos);
+      }
+      const int p = warp_append(take, &s_cnt[0]);
+      if (p >= 0 && base_out + p < (uint32_t)pl.k_max) out[base_out + p] = pos;
+    }
+  } else {
+    for_each_candidate(overflow, rc, n_stored, rs, n, (uint32_t)b1,
+                       [&](bool v, uint32_t key, int pos) {
+                         const bool pre = v && (int)((key >> 8) & 0xfffu) == b2;
+                         const int low = (int)(key & 0xffu);
+                         const bool take = pre && (low > b3 || (low == b3 && pos <= max_tie_pos));
+                         const int p = warp_append(take, &s_cnt[0]);
+                         if (p >= 0 && base_out + p < (uint32_t)pl.k_max) out[base_out + p] = pos;
+                       });
+  }
   __syncthreads();
   if (tid == 0) {
     sel_count[row] = k;
     kth[row] = key_score(kstar);
-    __threadfence();
-    if ((int)atomicAdd(n_out, 0u) != k) atomicOr(status, 1);
+    if ((int)(base_out + s_cnt[0]) != k) atomicOr(status, 1);
   }
 }
 

@@ -23,7 +23,7 @@ BUF_LUT, BUF_COARSE, BUF_SCORES, BUF_LIST_PARTIALS, BUF_SEL_IDX, BUF_SEL_COUNT, 
 EXPORTS = [
     "pqhsa_heads_per_group", "pqhsa_num_partials", "pqhsa_buffer_elems", "pqhsa_workspace_bytes",
     "pqhsa_build_lut", "pqhsa_scan", "pqhsa_select", "pqhsa_hybrid_attend", "pqhsa_decode",
-    "pqhsa_decode_host", "pqhsa_last_device_status", "pqhsa_decode_buffer_offset",
+    "pqhsa_decode_events", "pqhsa_decode_host", "pqhsa_last_device_status", "pqhsa_decode_buffer_offset",
     "pqhsa_decode_launch_count", "pqhsa_status_string",
 ]
 
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
             "pqhsa_select": (I, [P, V, V, V, V, V, V, Z, V]),
             "pqhsa_hybrid_attend": (I, [P, V, PK, PI, V, V, V, V, V, V, V, V, Z, V]),
             "pqhsa_decode": (I, [P, V, PI, PK, V, V, V, Z, V]),
+            "pqhsa_decode_events": (I, [P, V, PI, PK, V, V, V, Z, V, ctypes.POINTER(V)]),
             "pqhsa_decode_host": (I, [P, V, V, PI, PK, V, V, V, V, Z, V]),
             "pqhsa_last_device_status": (I, [P, V, V]),
             "pqhsa_decode_buffer_offset": (Z, [P, I]),
@@ -195,6 +196,18 @@ def decode(params, q, index: Index, kv: PagedKV, seq_lens, out, ws, stream=None)
     _check("pqhsa_decode", lib().pqhsa_decode(
         ctypes.byref(params), _ptr(q), ctypes.byref(index), ctypes.byref(kv), _ptr(seq_lens),
         _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+N_STAGE_EVENTS = 5
+
+
+def decode_events(params, q, index: Index, kv: PagedKV, seq_lens, out, ws, events, stream=None) -> None:
+    """`events`: five torch.cuda.Event(enable_timing=True) that have been recorded once (so
+    that their CUDA handles exist); the library re-records them around its stages."""
+    arr = (ctypes.c_void_p * N_STAGE_EVENTS)(*[e.cuda_event for e in events])
+    _check("pqhsa_decode_events", lib().pqhsa_decode_events(
+        ctypes.byref(params), _ptr(q), ctypes.byref(index), ctypes.byref(kv), _ptr(seq_lens),
+        _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream), arr))
 
 
 def decode_host(params, q_host, q_staging, index: Index, kv: PagedKV, seq_lens, out_staging,

@@ -9,8 +9,10 @@ from paper_2609_33746_b200.index_builder import build_index
 from paper_2609_33746_b200.workload import DecodeConfig, generate
 
 
-def make_case(cfg: DecodeConfig, device="cpu"):
+def make_case(cfg: DecodeConfig, device="cpu", pre_index=None):
     inp = generate(cfg, device=device)
+    if pre_index is not None:
+        pre_index(inp)
     idx = build_index(inp)
     return inp, idx
 

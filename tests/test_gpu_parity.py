@@ -55,14 +55,32 @@ CASES = {
     "full_budget": small("full", seq_lens=(700,), budget_ppm=1000000, n_q_heads=4, n_kv_heads=1),
     "many_lists": small("lists", seq_lens=(6000,), n_list=1024, n_q_heads=4, n_kv_heads=1,
                         kmeans_iters=2),
+    # logits of late tokens exceed those of the first tiles by far more than exp can hold:
+    # the scan must rebuild its per-list sums against the true maximum
+    "norm_jump": small("jump", seq_lens=(40000,), n_q_heads=4, n_kv_heads=1, kmeans_iters=1),
+    "odd_list_count": small("odd", seq_lens=(1000,), n_list=37, n_q_heads=2, n_kv_heads=2,
+                            kmeans_iters=1),
 }
+
+
+def _norm_jump(inp):
+    """Scale the cached keys (powers of two: exact in bf16) before the index is built."""
+    first_late_page = 30000 // inp.cfg.page_size
+    n_pages = (inp.cfg.seq_lens[0] + inp.cfg.page_size - 1) // inp.cfg.page_size
+    early = inp.block_table[0, :first_late_page].long()
+    late = inp.block_table[0, first_late_page:n_pages].long()
+    inp.k_cache[early] *= 0.25
+    inp.k_cache[late] *= 2.0
+
+
+PRE = {"norm_jump": _norm_jump}
 
 _cache = {}
 
 
 def get_case(key):
     if key not in _cache:
-        inp, idx = make_case(CASES[key], device="cuda")
+        inp, idx = make_case(CASES[key], device="cuda", pre_index=PRE.get(key))
         arrays = oracle_arrays(inp, idx)
         ref = run_oracle(inp, idx, arrays=arrays)
         op = DecodeOp(inp, idx)

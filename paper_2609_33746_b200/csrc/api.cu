@@ -72,9 +72,14 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.upb = o.Hkv * o.n_hg;
   o.n_part = o.scan_ctas / o.upb + 2;
   o.rows = o.B * o.Hq;
-  // the coarse table is bulk-copied: its byte size and unit stride must be multiples of 16
-  if (scan_smem_bytes(o, true) <= kMaxSmemPerCta && (o.Gc * o.n_list) % 4 == 0) o.coarse_in_smem = 1;
-  else if (scan_smem_bytes(o, false) <= kMaxSmemPerCta) o.coarse_in_smem = 0;
+  // the coarse table is bulk-copied: its byte size and unit stride must be multiples of 16.
+  // Prefer a 3-stage code ring with the coarse table in shared memory, then give up the
+  // coarse table, then a stage.
+  const bool co_ok = (o.Gc * o.n_list) % 4 == 0;
+  if (co_ok && scan_smem_bytes(o, true, 3) <= kMaxSmemPerCta) { o.coarse_in_smem = 1; o.scan_stages = 3; }
+  else if (scan_smem_bytes(o, false, 3) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 3; }
+  else if (co_ok && scan_smem_bytes(o, true, 2) <= kMaxSmemPerCta) { o.coarse_in_smem = 1; o.scan_stages = 2; }
+  else if (scan_smem_bytes(o, false, 2) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 2; }
   else return PQHSA_ERR_UNSUPPORTED;
 
   o.hist_chunks = ceil_div(o.N_max, kSelChunk);

@@ -14,14 +14,17 @@ namespace pqhsa {
 constexpr int kHeadDim = 128;
 constexpr int kNCode = 256;
 constexpr int kTile = 32;            // tokens per scan tile: one token per lane
-constexpr int kScanThreads = 512;
+#ifndef PQHSA_SCAN_THREADS
+#define PQHSA_SCAN_THREADS 512
+#endif
+constexpr int kScanThreads = PQHSA_SCAN_THREADS;
 constexpr int kScanMinTiles = kScanThreads / 32;   // a scan CTA gets at least one tile per warp
 constexpr int kHistBins = 4096;      // 12-bit radix digits for the two coarse select levels
 constexpr int kSelThreads = 512;
 constexpr int kSelChunk = 8192;      // scores per select CTA: 16 per thread, kept in registers
 constexpr int kAttendThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kNegligibleLog2 = -64.0f;   // exp2 arguments below this add nothing to a sum
+constexpr float kNegligibleLog2 = -40.0f;   // exp2 arguments below this are left out of a sum
 
 // Host-derived launch plan; passed by value to kernels.
 struct Plan {
@@ -40,6 +43,7 @@ struct Plan {
   int cand_cap;                      // candidate slots per row
   int splits;                        // split-K CTAs per row in the attend kernel
   int coarse_in_smem;                // scan keeps the coarse table in shared memory
+  int scan_stages;                   // cp.async stages per warp in the scan's code ring (3 or 2)
   int num_sms;
 };
 
@@ -149,6 +153,6 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
                           const float* list_partials, const int32_t* sel_idx,
                           const int32_t* sel_count, const int32_t* seq_lens, void* out,
                           float* lse, cudaStream_t st);
-size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem);
+size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem, int stages);
 
 }  // namespace pqhsa

@@ -10,6 +10,12 @@
 // positions static each lane permutes its own code bytes once per token
 // (byte p <- byte p ^ (lane & 7)).
 //
+// The codes stream from HBM through a per-warp ring of cp.async stages in shared memory
+// (kStages tiles of 32 tokens in flight per warp), so the bytes in flight do not depend on
+// registers; 16-byte chunks are placed with an XOR swizzle that makes the lane-per-token
+// 16-byte reads conflict free as well.  Norms and list ids (6 bytes per token) are
+// prefetched one tile ahead in registers.
+//
 // Per-list exp-sums: the CTA takes the maximum logit of its first round of tiles (one tile
 // per warp) as reference and adds exp(l~ - ref) into a [Gc][n_list] table in shared memory
 // while it scans.  When the segment is done the sums are re-based to the segment's true
@@ -20,54 +26,136 @@
 
 namespace pqhsa {
 
-template <int GC> struct VecT;
-template <> struct VecT<1> { using type = float; };
-template <> struct VecT<2> { using type = float2; };
-template <> struct VecT<4> { using type = float4; };
+// Packed accumulators: the Gc partial sums of a token live in 64-bit registers holding two
+// floats each, so one table entry is added with add.f32x2 (two lanes per instruction).
+template <int GC> struct Acc;
+template <> struct Acc<4> {
+  unsigned long long lo, hi;
+  __device__ __forceinline__ void zero() { lo = 0ull; hi = 0ull; }
+  __device__ __forceinline__ void load(uint32_t saddr) {
+    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(lo), "=l"(hi) : "r"(saddr));
+  }
+  __device__ __forceinline__ void merge(const Acc& o) {
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(lo) : "l"(o.lo));
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(hi) : "l"(o.hi));
+  }
+  __device__ __forceinline__ void get(float (&f)[4]) const {
+    f[0] = __uint_as_float((uint32_t)lo); f[1] = __uint_as_float((uint32_t)(lo >> 32));
+    f[2] = __uint_as_float((uint32_t)hi); f[3] = __uint_as_float((uint32_t)(hi >> 32));
+  }
+};
+template <> struct Acc<2> {
+  unsigned long long lo;
+  __device__ __forceinline__ void zero() { lo = 0ull; }
+  __device__ __forceinline__ void load(uint32_t saddr) {
+    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(lo) : "r"(saddr));
+  }
+  __device__ __forceinline__ void merge(const Acc& o) {
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(lo) : "l"(o.lo));
+  }
+  __device__ __forceinline__ void get(float (&f)[2]) const {
+    f[0] = __uint_as_float((uint32_t)lo); f[1] = __uint_as_float((uint32_t)(lo >> 32));
+  }
+};
+template <> struct Acc<1> {
+  float v;
+  __device__ __forceinline__ void zero() { v = 0.f; }
+  __device__ __forceinline__ void load(uint32_t saddr) {
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(saddr));
+  }
+  __device__ __forceinline__ void merge(const Acc& o) { v += o.v; }
+  __device__ __forceinline__ void get(float (&f)[1]) const { f[0] = v; }
+};
 
-template <int GC> __device__ __forceinline__ void vec_add(float (&acc)[GC],
-                                                          const typename VecT<GC>::type& v);
-template <> __device__ __forceinline__ void vec_add<1>(float (&a)[1], const float& v) { a[0] += v; }
-template <> __device__ __forceinline__ void vec_add<2>(float (&a)[2], const float2& v) {
-  a[0] += v.x; a[1] += v.y;
+template <int GC> __device__ __forceinline__ void load_vec(float (&f)[GC], const float* p);
+template <> __device__ __forceinline__ void load_vec<1>(float (&f)[1], const float* p) { f[0] = *p; }
+template <> __device__ __forceinline__ void load_vec<2>(float (&f)[2], const float* p) {
+  const float2 v = *reinterpret_cast<const float2*>(p);
+  f[0] = v.x; f[1] = v.y;
 }
-template <> __device__ __forceinline__ void vec_add<4>(float (&a)[4], const float4& v) {
-  a[0] += v.x; a[1] += v.y; a[2] += v.z; a[3] += v.w;
+template <> __device__ __forceinline__ void load_vec<4>(float (&f)[4], const float* p) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
 }
 
 constexpr float kOverflowGuardLog2 = 96.0f;   // exp2 arguments above this trigger the rebuild
 constexpr int kMbarSpinLimit = 1 << 22;
 
-template <int M> struct TokenRec {
-  uint32_t w[M / 4];   // code bytes
+struct TokenMeta {
   float norm;          // r_i
   uint32_t lid;        // a_i
 };
 
-template <int M>
-__device__ __forceinline__ void load_token(TokenRec<M>& r, const uint8_t* __restrict__ codes,
-                                           const uint16_t* __restrict__ lids,
-                                           const float* __restrict__ norms, size_t row_base,
-                                           int i, bool valid) {
+__device__ __forceinline__ void load_meta(TokenMeta& r, const uint16_t* __restrict__ lids,
+                                          const float* __restrict__ norms, size_t row_base, int i,
+                                          bool valid) {
+  r.lid = 0u;
+  r.norm = 0.f;
   if (valid) {
-    const uint8_t* p = codes + (row_base + i) * M;
-    if constexpr (M == 8) {
-      uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
-      r.w[0] = v.x; r.w[1] = v.y;
-    } else {
-#pragma unroll
-      for (int c = 0; c < M / 16; ++c) {
-        uint4 v = __ldg(reinterpret_cast<const uint4*>(p) + c);
-        r.w[4 * c + 0] = v.x; r.w[4 * c + 1] = v.y; r.w[4 * c + 2] = v.z; r.w[4 * c + 3] = v.w;
-      }
-    }
     r.lid = __ldg(lids + row_base + i);
     r.norm = norms ? __ldg(norms + row_base + i) : 1.0f;
+  }
+}
+
+// ---- per-warp cp.async ring for the code tiles
+template <int M> struct CodeTile {
+  static constexpr int kChunkBytes = M < 16 ? M : 16;       // one cp.async
+  static constexpr int kChunksPerToken = M / kChunkBytes;   // C
+  static constexpr int kChunks = kTile * kChunksPerToken;
+  static constexpr int kBytes = kTile * M;
+  // chunk c of token tok sits at chunk slot c ^ swz(tok): lanes of a quarter warp then read
+  // eight different 16-byte bank groups
+  static __device__ __forceinline__ int swz(int tok) {
+    return (tok * kChunksPerToken >> 3) & (kChunksPerToken - 1);
+  }
+};
+
+__device__ __forceinline__ void cp_async(uint32_t dst, const void* src, int bytes16) {
+  if (bytes16)
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+  else
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() {
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Issues the copies of tile t (tokens t*32 .. t*32+31 of the row) into a ring slot.
+template <int M>
+__device__ __forceinline__ void issue_tile(uint32_t slot, const uint8_t* __restrict__ codes,
+                                           size_t row_base, int t, int tend, int Nb, int lane) {
+  using CT = CodeTile<M>;
+  if (t < tend) {
+#pragma unroll
+    for (int q0 = 0; q0 < CT::kChunks; q0 += 32) {
+      const int q = q0 + lane;
+      const int tok = q / CT::kChunksPerToken, c = q % CT::kChunksPerToken;
+      const int i = t * kTile + tok;
+      if (i < Nb)
+        cp_async(slot + tok * M + ((c ^ CT::swz(tok)) * CT::kChunkBytes),
+                 codes + (row_base + i) * M + c * CT::kChunkBytes, CT::kChunkBytes == 16);
+    }
+  }
+  cp_async_commit();
+}
+
+// This lane's token: its code bytes from the ring slot, 4 per register, in original order.
+template <int M>
+__device__ __forceinline__ void read_codes(uint32_t slot, int lane, uint32_t (&w)[M / 4]) {
+  using CT = CodeTile<M>;
+  const uint32_t tok_addr = slot + lane * M;
+  if constexpr (M == 8) {
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(tok_addr));
   } else {
 #pragma unroll
-    for (int c = 0; c < M / 4; ++c) r.w[c] = 0u;
-    r.lid = 0u;
-    r.norm = 0.f;
+    for (int c = 0; c < CT::kChunksPerToken; ++c) {
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3])
+                   : "r"(tok_addr + ((c ^ CT::swz(lane)) * 16)));
+    }
   }
 }
 
@@ -101,23 +189,30 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return false;
 }
 
-template <int M, int GC>
+template <int M, int GC, int kStages>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restrict__ lids,
             const float* __restrict__ norms, const float* __restrict__ lut,
             const float* __restrict__ coarse, const int32_t* __restrict__ seq_lens,
             float* __restrict__ scores, float* __restrict__ partials, int* __restrict__ status) {
-  using Vec = typename VecT<GC>::type;
   constexpr int kLutFloats = kNCode * M * GC;
   constexpr int kEntryBytes = GC * 4;
   constexpr int kRowBytes = M * kEntryBytes;       // stride between consecutive z
   constexpr int kWarps = kScanThreads / 32;
-  constexpr int kBlk = 8;                          // table reads issued back to back
+#ifndef PQHSA_SCAN_BLK
+#define PQHSA_SCAN_BLK 8
+#endif
+  constexpr int kBlk = PQHSA_SCAN_BLK;             // table reads issued back to back
 
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* s_lut = reinterpret_cast<float*>(smem_raw);
   float* s_sums = s_lut + kLutFloats;                       // [GC][n_list]
   float* s_coarse = s_sums + GC * pl.n_list;                // [n_list][GC] when it fits
+  // the code ring sits behind the tables: kStages tiles per warp
+  const uint32_t table_bytes =
+      uint32_t(kLutFloats + GC * pl.n_list * (pl.coarse_in_smem ? 2 : 1)) * 4u;
+  const uint32_t ring0 = smem_u32(smem_raw) + ((table_bytes + 127u) & ~127u) +
+                         uint32_t((threadIdx.x >> 5) * kStages * CodeTile<M>::kBytes);
   __shared__ float s_red[kWarps][GC];
   __shared__ float s_ref[GC], s_max[GC];
   __shared__ int s_overflow;
@@ -146,10 +241,9 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   const int lx = lane & 7;
   const uint32_t byte_sel = 0x3210u ^ (uint32_t(lane & 3) * 0x1111u);
   const bool swap_words = (lane & 4) != 0;
-  const unsigned char* lut_bytes = reinterpret_cast<const unsigned char*>(s_lut);
-  uint32_t lane_off[8];   // byte offset of entry (z = 0, m = t ^ lx) for t = s & 7
+  uint32_t lane_off[8];   // shared-window address of entry (z = 0, m = t ^ lx) for t = s & 7
 #pragma unroll
-  for (int t = 0; t < 8; ++t) lane_off[t] = uint32_t((t ^ lx) * kEntryBytes);
+  for (int t = 0; t < 8; ++t) lane_off[t] = smem_u32(s_lut) + uint32_t((t ^ lx) * kEntryBytes);
 
   // locate the sequence that holds tile `lo`
   int b = 0;
@@ -188,11 +282,14 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     }
     for (int i = tid; i < GC * n_list; i += kScanThreads) s_sums[i] = 0.f;
 
-    // first tile of this warp: its global loads overlap the table copy
+    // prologue of the ring: the first kStages-1 tiles of this warp (overlaps the table copy)
     int t = t0 + warp;
-    TokenRec<M> cur;
-    load_token<M>(cur, codes, lids, norms, row_base, t * kTile + lane,
-                  t < tend && t * kTile + lane < Nb);
+#pragma unroll
+    for (int st = 0; st < kStages - 1; ++st)
+      issue_tile<M>(ring0 + st * CodeTile<M>::kBytes, codes, row_base, t + st * kWarps, tend, Nb,
+                    lane);
+    TokenMeta cur;
+    load_meta(cur, lids, norms, row_base, t * kTile + lane, t < tend && t * kTile + lane < Nb);
     if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, 4);
     bar_parity ^= 1u;
     __syncthreads();   // s_sums zeroed, tables landed
@@ -202,13 +299,17 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     for (int g = 0; g < GC; ++g) { mx[g] = -CUDART_INF_F; ref2[g] = 0.f; }
     bool first = true;
     bool more = true;
+    int it = 0;
     while (more) {
       const bool have = t < tend;
       const int tn = t + kWarps;
-      TokenRec<M> nxt = cur;
-      if (have && tn < tend)
-        load_token<M>(nxt, codes, lids, norms, row_base, tn * kTile + lane,
-                      tn * kTile + lane < Nb);
+      __syncwarp();      // every lane is done reading the slot that is refilled next
+      issue_tile<M>(ring0 + ((it + kStages - 1) % kStages) * CodeTile<M>::kBytes, codes, row_base,
+                    t + (kStages - 1) * kWarps, tend, Nb, lane);
+      TokenMeta nxt;
+      load_meta(nxt, lids, norms, row_base, tn * kTile + lane, tn < tend && tn * kTile + lane < Nb);
+      cp_async_wait<kStages - 1>();
+      __syncwarp();      // the copies of all lanes for tile t have landed
       const int i = t * kTile + lane;
       const bool valid = have && i < Nb;
       float sc[GC];
@@ -217,45 +318,42 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
 
       if (have) {
         // position p of the lane's code array <- original byte p ^ (lane & 7)
-        uint32_t cw[M / 4];
+        uint32_t raw[M / 4], cw[M / 4];
+        read_codes<M>(ring0 + (it % kStages) * CodeTile<M>::kBytes, lane, raw);
 #pragma unroll
         for (int j = 0; j < M / 8; ++j) {
-          const uint32_t a = cur.w[2 * j], bb = cur.w[2 * j + 1];
+          const uint32_t a = raw[2 * j], bb = raw[2 * j + 1];
           cw[2 * j] = __byte_perm(swap_words ? bb : a, 0u, byte_sel);
           cw[2 * j + 1] = __byte_perm(swap_words ? a : bb, 0u, byte_sel);
         }
-        float acc0[GC], acc1[GC];
-#pragma unroll
-        for (int g = 0; g < GC; ++g) { acc0[g] = 0.f; acc1[g] = 0.f; }
+        Acc<GC> acc0, acc1;
+        acc0.zero();
+        acc1.zero();
 #pragma unroll
         for (int sb = 0; sb < M; sb += kBlk) {
-          Vec v[kBlk];
+          Acc<GC> v[kBlk];
 #pragma unroll
           for (int u = 0; u < kBlk; ++u) {
             const int s = sb + u;
             const uint32_t z = __byte_perm(cw[s >> 2], 0u, 0x4440u | uint32_t(s & 3));
-            const uint32_t off = lane_off[s & 7] + z * uint32_t(kRowBytes) +
-                                 uint32_t((s & ~7) * kEntryBytes);
-            v[u] = *reinterpret_cast<const Vec*>(lut_bytes + off);
+            v[u].load(lane_off[s & 7] + z * uint32_t(kRowBytes) + uint32_t((s & ~7) * kEntryBytes));
           }
 #pragma unroll
           for (int u = 0; u < kBlk; u += 2) {
-            vec_add<GC>(acc0, v[u]);
-            vec_add<GC>(acc1, v[u + 1]);
+            acc0.merge(v[u]);
+            acc1.merge(v[u + 1]);
           }
         }
-        float co[GC];
-#pragma unroll
-        for (int g = 0; g < GC; ++g) co[g] = 0.f;
-        if (pl.coarse_in_smem)
-          vec_add<GC>(co, *reinterpret_cast<const Vec*>(s_coarse + cur.lid * GC));
-        else
-          vec_add<GC>(co, __ldg(reinterpret_cast<const Vec*>(g_coarse + cur.lid * GC)));
+        acc0.merge(acc1);
+        float accf[GC], co[GC];
+        acc0.get(accf);
+        if (pl.coarse_in_smem) load_vec<GC>(co, s_coarse + cur.lid * GC);
+        else load_vec<GC>(co, g_coarse + cur.lid * GC);
         if (valid) {
 #pragma unroll
           for (int g = 0; g < GC; ++g) {
             if (g < n_heads) {
-              sc[g] = cur.norm * (co[g] + (acc0[g] + acc1[g]));
+              sc[g] = cur.norm * (co[g] + accf[g]);
               scores[(size_t)(row0 + g) * N_max + i] = sc[g];
               mx[g] = fmaxf(mx[g], sc[g]);
             }
@@ -282,22 +380,30 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         first = false;
       }
       if (valid) {
-        bool over = false;
+        float x[GC], xm = -CUDART_INF_F;
 #pragma unroll
         for (int g = 0; g < GC; ++g) {
-          if (g < n_heads) {
-            const float x = fmaf(sc[g], kLog2e, -ref2[g]);
-            if (x > kOverflowGuardLog2) over = true;
-            else if (x > kNegligibleLog2) atomicAdd(&s_sums[g * n_list + cur.lid], fast_exp2(x));
+          x[g] = fmaf(sc[g], kLog2e, -ref2[g]);      // -inf for padded head slots
+          xm = fmaxf(xm, x[g]);
+        }
+        if (xm > kNegligibleLog2) {
+          if (xm > kOverflowGuardLog2) {
+            s_overflow = 1;
+          } else {
+#pragma unroll
+            for (int g = 0; g < GC; ++g)
+              if (x[g] > kNegligibleLog2)
+                atomicAdd(&s_sums[g * n_list + cur.lid], fast_exp2(x[g]));
           }
         }
-        if (over) s_overflow = 1;
       }
       cur = nxt;
       t = tn;
+      ++it;
       more = t < tend;
     }
 
+    cp_async_wait<0>();
     // segment maximum per head
     __syncthreads();   // s_red free again, all table updates done
 #pragma unroll
@@ -351,21 +457,22 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   }
 }
 
-size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem) {
+size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem, int stages) {
   size_t f = (size_t)kNCode * pl.M * pl.Gc + (size_t)pl.Gc * pl.n_list;
   if (coarse_in_smem) f += (size_t)pl.Gc * pl.n_list;
-  return f * sizeof(float);
+  const size_t tables = (f * sizeof(float) + 127) / 128 * 128;    // the ring is 128-byte aligned
+  return tables + (size_t)(kScanThreads / 32) * stages * kTile * pl.M;
 }
 
-template <int M, int GC>
+template <int M, int GC, int S>
 static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const float* lut,
                                  const float* coarse, const int32_t* seq_lens, float* scores,
                                  float* partials, int* status, cudaStream_t st) {
-  const size_t smem = scan_smem_bytes(pl, pl.coarse_in_smem != 0);
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC>,
+  const size_t smem = scan_smem_bytes(pl, pl.coarse_in_smem != 0, S);
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  scan_kernel<M, GC><<<pl.scan_ctas, kScanThreads, smem, st>>>(
+  scan_kernel<M, GC, S><<<pl.scan_ctas, kScanThreads, smem, st>>>(
       pl, ix.codes, ix.list_ids, ix.key_norms, lut, coarse, seq_lens, scores, partials, status);
   return cudaGetLastError();
 }
@@ -373,9 +480,14 @@ static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const fl
 cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,
                         const float* coarse, const int32_t* seq_lens, float* scores,
                         float* list_partials, int* status, cudaStream_t st) {
-#define PQHSA_SCAN_CASE(MM, GG)                                                              \
-  if (pl.M == MM && pl.Gc == GG)                                                             \
-    return launch_scan_t<MM, GG>(pl, ix, lut, coarse, seq_lens, scores, list_partials, status, st);
+#define PQHSA_SCAN_CASE(MM, GG)                                                               \
+  if (pl.M == MM && pl.Gc == GG) {                                                            \
+    if (pl.scan_stages >= 3)                                                                  \
+      return launch_scan_t<MM, GG, 3>(pl, ix, lut, coarse, seq_lens, scores, list_partials,   \
+                                      status, st);                                            \
+    return launch_scan_t<MM, GG, 2>(pl, ix, lut, coarse, seq_lens, scores, list_partials,     \
+                                    status, st);                                              \
+  }
   PQHSA_SCAN_CASE(8, 1) PQHSA_SCAN_CASE(8, 2) PQHSA_SCAN_CASE(8, 4)
   PQHSA_SCAN_CASE(16, 1) PQHSA_SCAN_CASE(16, 2) PQHSA_SCAN_CASE(16, 4)
   PQHSA_SCAN_CASE(32, 1) PQHSA_SCAN_CASE(32, 2) PQHSA_SCAN_CASE(32, 4)

@@ -82,18 +82,25 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   else if (scan_smem_bytes(o, false, 2) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 2; }
   else return PQHSA_ERR_UNSUPPORTED;
 
-  o.hist_chunks = ceil_div(o.N_max, kSelChunk);
+  // select CTAs per row: enough CTAs to fill the GPU about twice over, each looping over
+  // 8192-score chunks of its row
+  o.hist_chunks = ceil_div(4LL * o.num_sms, o.rows);
+  if (o.hist_chunks > ceil_div(o.N_max, kSelChunk)) o.hist_chunks = ceil_div(o.N_max, kSelChunk);
+  if (o.hist_chunks < 1) o.hist_chunks = 1;
   o.cand_cap = o.N_max / 4 > 4096 ? o.N_max / 4 : 4096;
   if (o.cand_cap > o.N_max) o.cand_cap = o.N_max;
-  // split-K CTAs per row: about 96 selected tokens each, but enough CTAs to fill the GPU
+  // split-K CTAs per row: about 256 selected tokens each, but enough CTAs to fill the GPU
   // when there are few rows, as long as every CTA keeps at least 32 units of work
-  o.splits = ceil_div(o.k_max, 96);
+  o.splits = ceil_div(o.k_max, 256);
   int fill = ceil_div(4LL * o.num_sms, o.rows);
   const int max_fill = (o.k_max + o.n_list / 4) / 32 > 0 ? (o.k_max + o.n_list / 4) / 32 : 1;
   if (fill > max_fill) fill = max_fill;
   if (o.splits < fill) o.splits = fill;
   if (o.splits > 64) o.splits = 64;
   if (o.splits < 1) o.splits = 1;
+  o.bg_ctas = ceil_div(2LL * o.num_sms, o.rows);
+  if (o.bg_ctas > 8) o.bg_ctas = 8;
+  if (o.bg_ctas < 1) o.bg_ctas = 1;
   return PQHSA_OK;
 }
 
@@ -120,10 +127,11 @@ void make_layout(const Plan& pl, WsLayout* L) {
   L->hist2 = take((size_t)pl.rows * kHistBins * 4);
   L->counters = take((size_t)pl.rows * 16);
   L->attend_tickets = take((size_t)pl.rows * 4);
+  L->bg_mass = take((size_t)pl.rows * pl.n_list * 4);
+  L->attend_zero_bytes = o - L->attend_tickets;
   L->zero_bytes = o - L->zero_begin;
   L->rowstate = take((size_t)pl.rows * 16);
   L->cand = take((size_t)pl.rows * pl.cand_cap * 8);
-  L->bg_mass = take((size_t)pl.rows * pl.n_list * 4);
   L->bg_max = take((size_t)pl.rows * 4);
   L->split_part = take((size_t)pl.rows * pl.splits * (2 + kHeadDim) * 4);
   L->stage_end = o;
@@ -293,7 +301,7 @@ int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_p
   if ((rc = check_ws(ws, ws_bytes, L.stage_end)) != PQHSA_OK) return rc;
   char* w = static_cast<char*>(ws);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaMemsetAsync(w + L.attend_tickets, 0, (size_t)pl.rows * 4, st) != cudaSuccess)
+  if (cudaMemsetAsync(w + L.attend_tickets, 0, L.attend_zero_bytes, st) != cudaSuccess)
     return PQHSA_ERR_CUDA;
   return cuda_status(launch_attend(pl, L, w, q, *kv, *index, scores, list_partials, sel_idx,
                                    sel_count, seq_lens, out, lse_or_null, st));

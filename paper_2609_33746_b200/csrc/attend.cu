@@ -16,33 +16,50 @@ namespace pqhsa {
 
 namespace {
 
-constexpr int kBgThreads = 512;
+constexpr int kBgThreads = 256;
 constexpr int kPartStride = 2 + kHeadDim;     // m, Z, N[128]
+constexpr int kMaxSeg = 160;                  // >= n_part for any plan (148 SMs / 1 unit + 2)
 
+// grid (bg_ctas, rows).  CTA c merges a slice of the lists and subtracts a slice of the
+// selected tokens; both go into bg_mass (zeroed by the caller) with float atomics, so the
+// CTAs of a row need no ordering.  A list's mass can come out slightly negative when its
+// members are all selected (rounding); the consumer clamps at 0.
 __global__ void __launch_bounds__(kBgThreads)
 bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restrict__ partials,
                const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_count,
                const uint16_t* __restrict__ lids, const int32_t* __restrict__ seq_lens,
                float* __restrict__ bg_mass, float* __restrict__ bg_max) {
-  extern __shared__ float s_dyn[];            // [n_list] sums, then [n_part] segment scales
-  float* s_tot = s_dyn;
-  float* s_scale = s_dyn + pl.n_list;
-  const int row = blockIdx.x, tid = threadIdx.x;
+  __shared__ float s_scale[kMaxSeg];
+  const int row = blockIdx.y, c = blockIdx.x, C = gridDim.x, tid = threadIdx.x;
   const int b = row / pl.Hq, h = row % pl.Hq;
   const int kv = h / pl.G, hg = (h % pl.G) / pl.Gc;
   const int n_list = pl.n_list;
   const int n = clamp_len(seq_lens[b], pl.N_max);
   float* mass = bg_mass + (size_t)row * n_list;
   if (n == 0) {
-    for (int j = tid; j < n_list; j += kBgThreads) mass[j] = 0.f;
-    if (tid == 0) bg_max[row] = -CUDART_INF_F;
+    if (c == 0 && tid == 0) bg_max[row] = -CUDART_INF_F;
     return;
   }
-  // the selected tokens' scores and list ids: issue these gathers first
+  // the selected tokens of this CTA's slice: start their gathers first
   const int cnt = sel_count[row];
+  const int tl = (int)((long long)c * cnt / C), th = (int)((long long)(c + 1) * cnt / C);
   const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
   const float* rs = scores + (size_t)row * pl.N_max;
   const uint16_t* rl = lids + ((size_t)b * pl.Hkv + kv) * pl.N_max;
+  constexpr int kSelPer = 4;
+  int idx[kSelPer];
+  float sc[kSelPer];
+  uint32_t li[kSelPer];
+#pragma unroll
+  for (int u = 0; u < kSelPer; ++u) {
+    const int t = tl + u * kBgThreads + tid;
+    idx[u] = t < th ? sel[t] : -1;
+  }
+#pragma unroll
+  for (int u = 0; u < kSelPer; ++u) {
+    sc[u] = idx[u] >= 0 ? rs[idx[u]] : 0.f;
+    li[u] = idx[u] >= 0 ? rl[idx[u]] : 0u;
+  }
 
   // which scan segments cover this row's unit
   const ScanSplit sp = scan_split(seq_lens, pl.B, pl.N_max, pl.upb, pl.scan_ctas);
@@ -51,7 +68,7 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   const int tb = seq_tiles(seq_lens, b, pl.N_max);
   const long long s_u = base + (long long)(kv * pl.n_hg + hg) * tb;
   const int c_first = split_cta_of(sp, s_u);
-  const int nseg = split_cta_of(sp, s_u + tb - 1) - c_first + 1;
+  const int nseg = min(kMaxSeg, split_cta_of(sp, s_u + tb - 1) - c_first + 1);
   const float* pr = partials + (size_t)row * pl.n_part * (n_list + 1);
 
   if (tid < nseg) s_scale[tid] = pr[(size_t)tid * (n_list + 1)];     // segment maxima
@@ -62,46 +79,34 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   __syncthreads();
   if (tid < nseg) s_scale[tid] = fast_exp2(fmaf(s_scale[tid], kLog2e, -m2));
   __syncthreads();
-  for (int j = tid; j < n_list; j += kBgThreads) {
+  const int jl = (int)((long long)c * n_list / C), jh = (int)((long long)(c + 1) * n_list / C);
+  for (int j = jl + tid; j < jh; j += kBgThreads) {
     float acc = 0.f;
-    int s = 0;
-    for (; s + 4 <= nseg; s += 4) {
-      float v[4];
+    for (int s0 = 0; s0 < nseg; s0 += 8) {
+      float v[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) v[u] = pr[(size_t)(s + u) * (n_list + 1) + 1 + j];
+      for (int u = 0; u < 8; ++u)
+        v[u] = (s0 + u < nseg) ? pr[(size_t)(s0 + u) * (n_list + 1) + 1 + j] : 0.f;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) acc = fmaf(v[u], s_scale[s + u], acc);
+      for (int u = 0; u < 8; ++u)
+        if (s0 + u < nseg) acc = fmaf(v[u], s_scale[s0 + u], acc);
     }
-    for (; s < nseg; ++s) acc = fmaf(pr[(size_t)s * (n_list + 1) + 1 + j], s_scale[s], acc);
-    s_tot[j] = acc;
+    if (acc != 0.f) atomicAdd(&mass[j], acc);
   }
-  __syncthreads();
   // take the selected tokens out of their lists' sums
-  for (int t0 = 0; t0 < cnt; t0 += kBgThreads * 2) {
-    int idx[2];
-    float sc[2];
-    uint32_t li[2];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int t = t0 + u * kBgThreads + tid;
-      idx[u] = t < cnt ? sel[t] : -1;
-    }
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      sc[u] = idx[u] >= 0 ? rs[idx[u]] : 0.f;
-      li[u] = idx[u] >= 0 ? rl[idx[u]] : 0u;
-    }
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (idx[u] >= 0) {
-        const float x = fmaf(sc[u], kLog2e, -m2);
-        if (x > kNegligibleLog2) atomicAdd(&s_tot[li[u]], -fast_exp2(x));
-      }
+  for (int u = 0; u < kSelPer; ++u) {
+    if (idx[u] >= 0) {
+      const float x = fmaf(sc[u], kLog2e, -m2);
+      if (x > kNegligibleLog2) atomicAdd(&mass[li[u]], -fast_exp2(x));
     }
   }
-  __syncthreads();
-  for (int j = tid; j < n_list; j += kBgThreads) mass[j] = fmaxf(s_tot[j], 0.f);
-  if (tid == 0) bg_max[row] = m;
+  for (int t = tl + kSelPer * kBgThreads + tid; t < th; t += kBgThreads) {
+    const int i = sel[t];
+    const float x = fmaf(rs[i], kLog2e, -m2);
+    if (x > kNegligibleLog2) atomicAdd(&mass[rl[i]], -fast_exp2(x));
+  }
+  if (c == 0 && tid == 0) bg_max[row] = m;
 }
 
 template <typename T> struct Unpack;
@@ -186,7 +191,7 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
     for (int j0 = a; j0 < e; j0 += 32) {
-      const float mine = (j0 + lane < e) ? mass[j0 + lane] : 0.f;
+      const float mine = (j0 + lane < e) ? fmaxf(mass[j0 + lane], 0.f) : 0.f;
       unsigned live = __ballot_sync(0xffffffffu, mine > 0.f);
       while (live) {
         int jj[4];
@@ -234,14 +239,16 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
 #pragma unroll
   for (int t = 0; t < 16; ++t) st.acc[t] = 0.f;
 
+  // page id of this lane's first token (second dependent load); later batches prefetch
+  // position and page one batch ahead, while the current batch's rows are in flight
+  int my_page = my_pos >= 0 ? __ldg(bt + my_pos / pl.page_size) : 0;
   for (int base = wl; base < wh; base += 32) {
-    if (base != wl) my_pos = (base + lane < wh) ? sel[base + lane] : -1;
     long long off = 0;
-    if (my_pos >= 0) {
-      const int page = __ldg(bt + my_pos / pl.page_size);
-      off = (long long)page * stride_page + (long long)(my_pos % pl.page_size) * stride_token +
+    if (my_pos >= 0)
+      off = (long long)my_page * stride_page + (long long)(my_pos % pl.page_size) * stride_token +
             (long long)kv * stride_head;
-    }
+    const int nxt_pos = (base + 32 + lane < wh) ? sel[base + 32 + lane] : -1;
+    int nxt_page = 0;
     const int nb = min(32, wh - base);
     for (int j0 = 0; j0 < nb; j0 += 4 * U) {
       uint4 kr[U][2], vr[U][2];
@@ -260,6 +267,7 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
           kr[u][0] = kr[u][1] = vr[u][0] = vr[u][1] = make_uint4(0u, 0u, 0u, 0u);
         }
       }
+      if (j0 == 0 && nxt_pos >= 0) nxt_page = __ldg(bt + nxt_pos / pl.page_size);
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         float kf[8];
@@ -293,6 +301,8 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
         }
       }
     }
+    my_pos = nxt_pos;
+    my_page = nxt_page;
   }
   // merge the 4 lane groups of the warp (lanes with equal gl own the same dims)
 #pragma unroll
@@ -378,7 +388,7 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
   float* bg_max = reinterpret_cast<float*>(ws + L.bg_max);
   float* split_part = reinterpret_cast<float*>(ws + L.split_part);
   uint32_t* tickets = reinterpret_cast<uint32_t*>(ws + L.attend_tickets);
-  bg_prep_kernel<<<pl.rows, kBgThreads, (pl.n_list + pl.n_part) * sizeof(float), st>>>(
+  bg_prep_kernel<<<dim3(pl.bg_ctas, pl.rows), kBgThreads, 0, st>>>(
       pl, scores, list_partials, sel_idx, sel_count, ix.list_ids, seq_lens, bg_mass, bg_max);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -39,9 +39,10 @@ struct Plan {
   int n_part;                        // list-partial slots per score row
   int upb;                           // scan units per sequence = Hkv * n_hg
   int rows;                          // B * Hq score rows
-  int hist_chunks;                   // CTAs per row in the select kernels: ceil(N_max / kSelChunk)
+  int hist_chunks;                   // CTAs per row in the select kernels
   int cand_cap;                      // candidate slots per row
   int splits;                        // split-K CTAs per row in the attend kernel
+  int bg_ctas;                       // CTAs per row in the background preparation
   int coarse_in_smem;                // scan keeps the coarse table in shared memory
   int scan_stages;                   // cp.async stages per warp in the scan's code ring (3 or 2)
   int num_sms;
@@ -54,9 +55,10 @@ struct WsLayout {
   size_t hist1, hist2;               // uint32 [rows][kHistBins] each
   size_t counters;                   // uint32 [rows][4]: ticket1, ticket2, n_out, n_cand
   size_t attend_tickets;             // uint32 [rows]
+  size_t attend_zero_bytes;          // tickets + bg_mass: what the attend stage needs cleared
   size_t rowstate;                   // int32  [rows][4]: b1, k1, k, n
   size_t cand;                       // uint2  [rows][cand_cap]: (key, position)
-  size_t bg_mass;                    // float  [rows][n_list]: M_j relative to bg_max
+  size_t bg_mass;                    // float  [rows][n_list]: M_j relative to bg_max (accumulated)
   size_t bg_max;                     // float  [rows]
   size_t split_part;                 // float  [rows][splits][2 + 128]: m, Z, N[128]
   size_t stage_end;                  // end of what a single stage call needs
@@ -71,8 +73,8 @@ void make_layout(const Plan& plan, WsLayout* L);
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ uint32_t score_key(float s) {
   // Order-preserving map float -> uint32 (larger score <-> larger key); -0 and +0 coincide.
-  uint32_t u = __float_as_uint(s + 0.0f);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  const uint32_t u = __float_as_uint(s + 0.0f);
+  return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
 }
 __device__ __forceinline__ float key_score(uint32_t k) {
   uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;

@@ -6,9 +6,10 @@
 // the layout the scan wants to find in shared memory: [z][m][g] with g the head inside its
 // head group, so one 16-byte read serves the four heads of a GQA group.
 //
-// The kernel is latency bound (a few MB of reads spread over the whole GPU), so every thread
-// issues all of its global loads (centroid rows, codewords) before the first use.  In the
-// fused decode call it also clears the counters and histograms that the top-k needs.
+// The kernel moves a few MB and is bound by latency and instruction issue, so every thread
+// issues its global loads (centroid rows, codeword) before the first use, the subspace
+// width is a template parameter, and four heads are reduced across a warp together.  In
+// the fused decode call it also clears the counters and histograms that the top-k needs.
 #include "common.cuh"
 
 namespace pqhsa {
@@ -25,18 +26,36 @@ template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16
   return __bfloat162float(v);
 }
 
-template <typename T>
+// Sums four per-lane values over the warp with 6 shuffles; afterwards every lane of the
+// 8-lane group g = lane >> 3 holds the total of value g.
+__device__ __forceinline__ float warp_sum4(float p0, float p1, float p2, float p3, int lane) {
+  const bool up16 = (lane & 16) != 0;
+  float keep0 = up16 ? p2 : p0, keep1 = up16 ? p3 : p1;
+  float send0 = up16 ? p0 : p2, send1 = up16 ? p1 : p3;
+  keep0 += __shfl_xor_sync(0xffffffffu, send0, 16);
+  keep1 += __shfl_xor_sync(0xffffffffu, send1, 16);
+  const bool up8 = (lane & 8) != 0;
+  float keep = up8 ? keep1 : keep0, send = up8 ? keep0 : keep1;
+  keep += __shfl_xor_sync(0xffffffffu, send, 8);
+  keep += __shfl_xor_sync(0xffffffffu, keep, 4);
+  keep += __shfl_xor_sync(0xffffffffu, keep, 2);
+  keep += __shfl_xor_sync(0xffffffffu, keep, 1);
+  return keep;
+}
+
+template <typename T, int DSUB>
 __global__ void __launch_bounds__(kLutThreads)
 build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ centroids,
                  const float* __restrict__ codebooks, float* __restrict__ lut,
                  float* __restrict__ coarse, uint4* __restrict__ zero_ptr, size_t zero_n16) {
-  __shared__ __align__(16) float sq[kMaxGroup][kHeadDim];   // sm_scale * q of the G heads
+  __shared__ __align__(16) float sq[kMaxGroup][kHeadDim];   // sm_scale * q of the heads, 0-padded
   const int kv = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = pl.G, Gc = pl.Gc, n_hg = pl.n_hg;
+  const int n_slots = n_hg * Gc;                            // head slots, >= G
   const size_t ukv = (size_t)b * pl.Hkv + kv;
 
-  // query -> shared (first dependent load of the kernel)
+  // query (first dependent load of the kernel)
   float qreg[(kMaxGroup * kHeadDim) / kLutThreads];
 #pragma unroll
   for (int u = 0; u < (kMaxGroup * kHeadDim) / kLutThreads; ++u) {
@@ -49,7 +68,8 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
   const int rows_per_cta = (pl.n_list + kLutChunks - 1) / kLutChunks;
   const int r0 = blockIdx.x * rows_per_cta;
   const int r1 = min(pl.n_list, r0 + rows_per_cta);
-  const int n_ent = pl.M * kNCode;
+  constexpr int kEntPerM = kNCode;
+  const int n_ent = pl.M * kEntPerM;
   const int ent_per_cta = (n_ent + kLutChunks - 1) / kLutChunks;
   const int e0 = blockIdx.x * ent_per_cta;
   const int e1 = min(n_ent, e0 + ent_per_cta);
@@ -62,13 +82,21 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
     if (j < r1)
       crow[u] = __ldg(reinterpret_cast<const float4*>(centroids + (ukv * pl.n_list + j) * kHeadDim) + lane);
   }
-  float cw[16];
-  {
-    const int e = e0 + tid;
-    const float* p = codebooks + (ukv * (size_t)n_ent + min(e, n_ent - 1)) * pl.dsub;
+  float cw[DSUB];
+  auto load_codeword = [&](int e) {
+    const float* p = codebooks + (ukv * (size_t)n_ent + e) * DSUB;
+    if constexpr (DSUB == 2) {
+      const float2 v = __ldg(reinterpret_cast<const float2*>(p));
+      cw[0] = v.x; cw[1] = v.y;
+    } else {
 #pragma unroll
-    for (int t = 0; t < 16; ++t) cw[t] = (t < pl.dsub && e < e1) ? __ldg(p + t) : 0.f;
-  }
+      for (int c = 0; c < DSUB / 4; ++c) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(p) + c);
+        cw[4 * c] = v.x; cw[4 * c + 1] = v.y; cw[4 * c + 2] = v.z; cw[4 * c + 3] = v.w;
+      }
+    }
+  };
+  if (e0 + tid < e1) load_codeword(e0 + tid);
 
   // ---- side job: clear a slice of the caller's zero region
   if (zero_ptr != nullptr) {
@@ -81,7 +109,7 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
 #pragma unroll
   for (int u = 0; u < (kMaxGroup * kHeadDim) / kLutThreads; ++u) {
     const int i = u * kLutThreads + tid;
-    if (i < G * kHeadDim) sq[i / kHeadDim][i % kHeadDim] = pl.sm_scale * qreg[u];
+    sq[i / kHeadDim][i % kHeadDim] = pl.sm_scale * qreg[u];      // rows >= G are zero
   }
   __syncthreads();
 
@@ -101,58 +129,69 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
       const int j = jb + warp + u * kLutWarps;
       if (j >= r1) continue;                       // warp-uniform
       const float4 c = crow[u];
-      for (int slot = 0; slot < n_hg * Gc; ++slot) {
-        float v = 0.f;
-        if (slot < G) {
-          const float4 qq = *reinterpret_cast<const float4*>(&sq[slot][4 * lane]);
-          v = warp_sum(c.x * qq.x + c.y * qq.y + c.z * qq.z + c.w * qq.w);
+      for (int hb = 0; hb < n_slots; hb += 4) {
+        float p[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const float4 qq = *reinterpret_cast<const float4*>(&sq[(hb + t) & (kMaxGroup - 1)][4 * lane]);
+          p[t] = c.x * qq.x + c.y * qq.y + c.z * qq.z + c.w * qq.w;
         }
-        if (lane == 0) {
-          int hg = slot / Gc, g = slot % Gc;
-          coarse[(((ukv * n_hg + hg) * pl.n_list) + j) * Gc + g] = v;
+        const float tot = warp_sum4(p[0], p[1], p[2], p[3], lane);
+        const int slot = hb + (lane >> 3);
+        if ((lane & 7) == 0 && slot < n_slots) {
+          const int hg = slot / Gc, g = slot % Gc;
+          coarse[(((ukv * n_hg + hg) * pl.n_list) + j) * Gc + g] = tot;
         }
       }
     }
   }
 
-  // ---- PQ table: one thread per (m, z); consecutive threads take consecutive z
+  // ---- PQ table: one thread per (m, z); consecutive threads take consecutive z, so the
+  //      subspace m (and with it the query sub-vector) is uniform over a warp
   for (int eb = e0; eb < e1; eb += kLutThreads) {
     const int e = eb + tid;
-    if (eb != e0 && e < e1) {
-      const float* p = codebooks + (ukv * (size_t)n_ent + e) * pl.dsub;
-#pragma unroll
-      for (int t = 0; t < 16; ++t) cw[t] = (t < pl.dsub) ? __ldg(p + t) : 0.f;
-    }
+    if (eb != e0 && e < e1) load_codeword(e);
     if (e >= e1) continue;
-    const int m = e / kNCode, z = e % kNCode;
+    const int m = e / kEntPerM, z = e % kEntPerM;
     for (int hg = 0; hg < n_hg; ++hg) {
-      float* dst = lut + (((ukv * n_hg + hg) * kNCode + z) * pl.M + m) * Gc;
-      for (int g = 0; g < Gc; ++g) {
-        const int h = hg * Gc + g;
-        float v = 0.f;
-        if (h < G) {
+      float v[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int t = 0; t < 16; ++t)
-            if (t < pl.dsub) v = fmaf(cw[t], sq[h][m * pl.dsub + t], v);
+      for (int g = 0; g < 4; ++g) {
+        if (g < Gc) {
+          const float* qs = &sq[(hg * Gc + g) & (kMaxGroup - 1)][m * DSUB];
+#pragma unroll
+          for (int t = 0; t < DSUB; ++t) v[g] = fmaf(cw[t], qs[t], v[g]);
         }
-        dst[g] = v;
       }
+      float* dst = lut + (((ukv * n_hg + hg) * kNCode + z) * pl.M + m) * Gc;
+      if (Gc == 4) *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+      else if (Gc == 2) *reinterpret_cast<float2*>(dst) = make_float2(v[0], v[1]);
+      else dst[0] = v[0];
     }
   }
 }
 
+template <typename T>
+static cudaError_t launch_lut_t(const Plan& pl, const T* q, const pqhsa_index& ix, float* lut,
+                                float* coarse, uint4* zp, size_t zn, cudaStream_t st) {
+  dim3 grid(kLutChunks, pl.Hkv, pl.B);
+  switch (pl.dsub) {
+    case 2: build_lut_kernel<T, 2><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
+    case 4: build_lut_kernel<T, 4><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
+    case 8: build_lut_kernel<T, 8><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
+    case 16: build_lut_kernel<T, 16><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
+}
+
 cudaError_t launch_build_lut(const Plan& pl, const void* q, const pqhsa_index& ix, float* lut,
                              float* coarse, void* zero_ptr, size_t zero_bytes, cudaStream_t st) {
-  dim3 grid(kLutChunks, pl.Hkv, pl.B);
   uint4* zp = static_cast<uint4*>(zero_ptr);
   const size_t zn = zero_bytes / 16;
   if (pl.dtype == PQHSA_F16)
-    build_lut_kernel<__half><<<grid, kLutThreads, 0, st>>>(
-        pl, static_cast<const __half*>(q), ix.centroids, ix.codebooks, lut, coarse, zp, zn);
-  else
-    build_lut_kernel<__nv_bfloat16><<<grid, kLutThreads, 0, st>>>(
-        pl, static_cast<const __nv_bfloat16*>(q), ix.centroids, ix.codebooks, lut, coarse, zp, zn);
-  return cudaGetLastError();
+    return launch_lut_t(pl, static_cast<const __half*>(q), ix, lut, coarse, zp, zn, st);
+  return launch_lut_t(pl, static_cast<const __nv_bfloat16*>(q), ix, lut, coarse, zp, zn, st);
 }
 
 }  // namespace pqhsa

@@ -131,15 +131,32 @@ sel_hist_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __rest
     return;
   }
   uint32_t* gh = hist1 + (size_t)row * kHistBins;
-  if (chunk * kSelChunk < n) {
-    float v[kElems];
-    int pos0[4];
-    load_chunk(scores + (size_t)row * pl.N_max, chunk, n, v, pos0);
+  const int n_chunks = (n + kSelChunk - 1) / kSelChunk;
+  if (chunk < n_chunks) {
+    const float* rs = scores + (size_t)row * pl.N_max;
+    float v[kElems], nv[kElems];
+    int pos0[4], npos0[4];
+    load_chunk(rs, chunk, n, v, pos0);
     for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
     __syncthreads();
+    for (int ch = chunk; ch < n_chunks; ch += gridDim.x) {
+      const bool more = ch + (int)gridDim.x < n_chunks;
+      if (more) load_chunk(rs, ch + gridDim.x, n, nv, npos0);     // in flight during the atomics
+      if ((ch + 1) * kSelChunk <= n) {               // full chunk: no bounds checks
 #pragma unroll
-    for (int e = 0; e < kElems; ++e)
-      if (pos0[e >> 2] + (e & 3) < n) atomicAdd(&s_hist[score_key(v[e]) >> 20], 1u);
+        for (int e = 0; e < kElems; ++e) atomicAdd(&s_hist[score_key(v[e]) >> 20], 1u);
+      } else {
+#pragma unroll
+        for (int e = 0; e < kElems; ++e)
+          if (pos0[e >> 2] + (e & 3) < n) atomicAdd(&s_hist[score_key(v[e]) >> 20], 1u);
+      }
+      if (more) {
+#pragma unroll
+        for (int e = 0; e < kElems; ++e) v[e] = nv[e];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) pos0[j] = npos0[j];
+      }
+    }
     __syncthreads();
     for (int i = tid; i < kHistBins; i += kSelThreads)
       if (s_hist[i]) atomicAdd(gh + i, s_hist[i]);
@@ -215,7 +232,7 @@ __device__ int block_count(int local, int* s_scan) {
   return tot;
 }
 
-__global__ void __launch_bounds__(kSelThreads)
+__global__ void __launch_bounds__(kSelThreads, 2)
 sel_filter_kernel(Plan pl, const float* __restrict__ scores, const uint32_t* __restrict__ hist1,
                   uint32_t* __restrict__ hist2, uint32_t* __restrict__ counters,
                   const int32_t* __restrict__ rowstate, uint2* __restrict__ cand,
@@ -225,7 +242,9 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, const uint32_t* __r
   __shared__ uint2 s_stash[kStashCap];
   __shared__ int s_scan[34];
   __shared__ int s_last;
-  __shared__ uint32_t s_base[2], s_cnt[2];
+  __shared__ uint32_t s_cnt[2];
+  __shared__ int s_scan2[2][32];
+  __shared__ uint32_t s_base2[2][2];
   const int row = blockIdx.y, tid = threadIdx.x, chunk = blockIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int b1 = rowstate[row * 4 + 0], k1 = rowstate[row * 4 + 1];
@@ -238,65 +257,83 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, const uint32_t* __r
   uint32_t* n_cand = &counters[row * 4 + 3];
   uint32_t* gh = hist2 + (size_t)row * kHistBins;
 
-  if (chunk * kSelChunk < n) {
-    float v[kElems];
-    int pos0[4];
+  const int n_chunks = (n + kSelChunk - 1) / kSelChunk;
+  if (chunk < n_chunks) {
+    float v[kElems], nv[kElems];
+    int pos0[4], npos0[4];
     load_chunk(rs, chunk, n, v, pos0);
     for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
+    // The key is monotone in the score, so "digit above / equal to b1" are two float
+    // compares: scores in [lo_f, hi_f] have top digit b1, scores above hi_f a larger one.
+    float lo_f = key_score((uint32_t)b1 << 20), hi_f = key_score(((uint32_t)b1 << 20) | 0xfffffu);
+    if (lo_f != lo_f) lo_f = -CUDART_INF_F;        // digit that starts inside the NaN patterns
     __syncthreads();
-    uint32_t keys[kElems];
-    uint32_t win_mask = 0, cand_mask = 0;
+    for (int ch = chunk; ch < n_chunks; ch += gridDim.x) {
+      const bool more = ch + (int)gridDim.x < n_chunks;
+      if (more) load_chunk(rs, ch + gridDim.x, n, nv, npos0);     // in flight during this chunk
+      uint32_t win_mask = 0, cand_mask = 0;
+      const bool full = (ch + 1) * kSelChunk <= n;
 #pragma unroll
-    for (int e = 0; e < kElems; ++e) {
-      keys[e] = score_key(v[e]);
-      const bool valid = pos0[e >> 2] + (e & 3) < n;
-      const int bin = (int)(keys[e] >> 20);
-      if (valid && bin > b1) win_mask |= 1u << e;
-      if (valid && bin == b1) {
-        cand_mask |= 1u << e;
-        atomicAdd(&s_hist[(keys[e] >> 8) & 0xfffu], 1u);
+      for (int e = 0; e < kElems; ++e) {
+        const bool valid = full || pos0[e >> 2] + (e & 3) < n;
+        const bool win = v[e] > hi_f;
+        const bool cnd = !win && v[e] >= lo_f;
+        if (valid && win) win_mask |= 1u << e;
+        if (valid && cnd) {
+          cand_mask |= 1u << e;
+          atomicAdd(&s_hist[(score_key(v[e]) >> 8) & 0xfffu], 1u);
+        }
       }
-    }
-    // exclusive scan of (winners << 16 | candidates) over the CTA
-    const uint32_t mine = ((uint32_t)__popc(win_mask) << 16) | (uint32_t)__popc(cand_mask);
-    uint32_t inc = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += u;
-    }
-    if (lane == 31) s_scan[warp] = (int)inc;
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t wv = (lane < kSelThreads / 32) ? (uint32_t)s_scan[lane] : 0u;
-      uint32_t ws = wv;
+      // exclusive scan of (winners << 16 | candidates) over the CTA
+      const uint32_t mine = ((uint32_t)__popc(win_mask) << 16) | (uint32_t)__popc(cand_mask);
+      uint32_t inc = mine;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t u = __shfl_up_sync(0xffffffffu, ws, o);
-        if (lane >= o) ws += u;
+        const uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += u;
       }
-      if (lane < kSelThreads / 32) s_scan[lane] = (int)(ws - wv);
-      if (lane == kSelThreads / 32 - 1) {        // CTA totals: take the output slots
-        const uint32_t tw = ws >> 16, tc = ws & 0xffffu;
-        s_base[0] = tw ? atomicAdd(n_out, tw) : 0u;
-        s_base[1] = tc ? atomicAdd(n_cand, tc) : 0u;
+      int* scan_buf = s_scan2[(ch / gridDim.x) & 1];     // two sets: no barrier to reuse them
+      uint32_t* base_buf = s_base2[(ch / gridDim.x) & 1];
+      if (lane == 31) scan_buf[warp] = (int)inc;
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t wv = (lane < kSelThreads / 32) ? (uint32_t)scan_buf[lane] : 0u;
+        uint32_t ws = wv;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t u = __shfl_up_sync(0xffffffffu, ws, o);
+          if (lane >= o) ws += u;
+        }
+        if (lane < kSelThreads / 32) scan_buf[16 + lane] = (int)(ws - wv);
+        if (lane == kSelThreads / 32 - 1) {        // CTA totals: take the output slots
+          const uint32_t tw = ws >> 16, tc = ws & 0xffffu;
+          base_buf[0] = tw ? atomicAdd(n_out, tw) : 0u;
+          base_buf[1] = tc ? atomicAdd(n_cand, tc) : 0u;
+        }
+      }
+      __syncthreads();
+      const uint32_t excl = (uint32_t)scan_buf[16 + warp] + inc - mine;
+      uint32_t pw = base_buf[0] + (excl >> 16), pc = base_buf[1] + (excl & 0xffffu);
+#pragma unroll
+      for (int e = 0; e < kElems; ++e) {
+        const int pos = pos0[e >> 2] + (e & 3);
+        if (win_mask & (1u << e)) {
+          if (pw < (uint32_t)pl.k_max) out[pw] = pos;
+          ++pw;
+        }
+        if (cand_mask & (1u << e)) {
+          if (pc < (uint32_t)pl.cand_cap) rc[pc] = make_uint2(score_key(v[e]), (uint32_t)pos);
+          ++pc;
+        }
+      }
+      if (more) {
+#pragma unroll
+        for (int e = 0; e < kElems; ++e) v[e] = nv[e];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) pos0[j] = npos0[j];
       }
     }
     __syncthreads();
-    const uint32_t excl = (uint32_t)s_scan[warp] + inc - mine;
-    uint32_t pw = s_base[0] + (excl >> 16), pc = s_base[1] + (excl & 0xffffu);
-#pragma unroll
-    for (int e = 0; e < kElems; ++e) {
-      const int pos = pos0[e >> 2] + (e & 3);
-      if (win_mask & (1u << e)) {
-        if (pw < (uint32_t)pl.k_max) out[pw] = pos;
-        ++pw;
-      }
-      if (cand_mask & (1u << e)) {
-        if (pc < (uint32_t)pl.cand_cap) rc[pc] = make_uint2(keys[e], (uint32_t)pos);
-        ++pc;
-      }
-    }
     for (int i = tid; i < kHistBins; i += kSelThreads)
       if (s_hist[i]) atomicAdd(gh + i, s_hist[i]);
     __threadfence();

@@ -151,6 +151,33 @@ int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_p
                         const int32_t* sel_count, const int32_t* seq_lens, void* out,
                         float* lse_or_null, void* ws, size_t ws_bytes, void* stream);
 
+/* pqhsa_select without a workspace argument.  (No counterpart in the paper: this entry point
+ * exists for integration, not for the method.)
+ *
+ * For callers that cannot allocate device memory where they need the top-k: code running
+ * inside an engine's pre-planned memory pool, plugins that receive tensors but no allocator,
+ * and paths where a driver allocation -- which may stall the whole device -- is not
+ * acceptable.  The scratch that pqhsa_select takes from `ws` (histograms, counters,
+ * candidate lists) lives instead in one fixed 16 MiB array inside the library image; every
+ * GPU that loads the library holds that array until the process exits.
+ *
+ *   - Same inputs, outputs and results as pqhsa_select.  Neither this call nor anything it
+ *     uses calls cudaMalloc, cudaFree or any allocating routine.
+ *   - Shapes whose scratch exceeds the array (pqhsa_select_static_bytes(params) >
+ *     pqhsa_select_static_capacity()) are rejected with PQHSA_ERR_WORKSPACE before anything
+ *     is launched; use pqhsa_select with your own workspace for those.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current).  Make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array and it keeps the last call's contents; each
+ *     call clears the part that must start at zero on `stream` first.  Two calls that can
+ *     overlap on the GPU (different streams, no dependency) race on it: serialise them.
+ *   - pqhsa_last_device_status does not apply; a count mismatch is not reported here. */
+size_t pqhsa_select_static_capacity(void);
+size_t pqhsa_select_static_bytes(const pqhsa_params* params);   /* 0 on invalid params */
+int pqhsa_select_static(const pqhsa_params* params, const float* scores, const int32_t* seq_lens,
+                        int32_t* sel_idx, int32_t* sel_count, float* kth_score, void* stream);
+
 /* Steps 1-4 back to back on one stream (Sec. 3.3: the decode step of one layer); all
  * intermediates live in `ws`. */
 int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* index,

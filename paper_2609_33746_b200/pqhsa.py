@@ -24,7 +24,8 @@ EXPORTS = [
     "pqhsa_heads_per_group", "pqhsa_num_partials", "pqhsa_buffer_elems", "pqhsa_workspace_bytes",
     "pqhsa_build_lut", "pqhsa_scan", "pqhsa_select", "pqhsa_hybrid_attend", "pqhsa_decode",
     "pqhsa_decode_events", "pqhsa_decode_host", "pqhsa_last_device_status", "pqhsa_decode_buffer_offset",
-    "pqhsa_decode_launch_count", "pqhsa_status_string",
+    "pqhsa_decode_launch_count", "pqhsa_status_string", "pqhsa_select_static",
+    "pqhsa_select_static_bytes", "pqhsa_select_static_capacity",
 ]
 
 
@@ -82,6 +83,9 @@ def lib() -> ctypes.CDLL:
             "pqhsa_decode_buffer_offset": (Z, [P, I]),
             "pqhsa_decode_launch_count": (I, [P]),
             "pqhsa_status_string": (ctypes.c_char_p, [I]),
+            "pqhsa_select_static": (I, [P, V, V, V, V, V, V]),
+            "pqhsa_select_static_bytes": (Z, [P]),
+            "pqhsa_select_static_capacity": (Z, []),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -182,6 +186,22 @@ def select(params, scores, seq_lens, sel_idx, sel_count, kth_score, ws, stream=N
     _check("pqhsa_select", lib().pqhsa_select(
         ctypes.byref(params), _ptr(scores), _ptr(seq_lens), _ptr(sel_idx), _ptr(sel_count),
         _ptr(kth_score), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def select_static_capacity() -> int:
+    return lib().pqhsa_select_static_capacity()
+
+
+def select_static_bytes(params: Params) -> int:
+    return lib().pqhsa_select_static_bytes(ctypes.byref(params))
+
+
+def select_static(params, scores, seq_lens, sel_idx, sel_count, kth_score, stream=None) -> None:
+    """pqhsa_select for callers that cannot allocate: the scratch is a fixed array inside the
+    library (shared by all calls on the device; shapes beyond its capacity are rejected)."""
+    _check("pqhsa_select_static", lib().pqhsa_select_static(
+        ctypes.byref(params), _ptr(scores), _ptr(seq_lens), _ptr(sel_idx), _ptr(sel_count),
+        _ptr(kth_score), _stream(stream)))
 
 
 def hybrid_attend(params, q, kv: PagedKV, index: Index, scores, list_partials, sel_idx, sel_count,

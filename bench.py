@@ -122,25 +122,10 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ oracle (CPU baseline / reference arm)
 def oracle_arrays_seq0(inp, idx):
-    """Float64 host copies of what the oracle needs for sequence 0: its index arrays and
-    its own KV pages, re-packed contiguously with an identity block table (a re-layout of
-    inputs; the oracle still reads rows through block table and strides)."""
-    import numpy as np
-    import torch
-    cfg = inp.cfg
-    assert cfg.kv_layout == "split"
-    f64 = lambda t: t.detach().cpu().double().numpy()
-    n = int(inp.seq_lens[0])
-    n_pages = max(1, (n + cfg.page_size - 1) // cfg.page_size)
-    pages = inp.block_table[0, :n_pages].long()
-    return dict(
-        q=f64(inp.q[:1]), centroids=f64(idx.centroids[:1]), codebooks=f64(idx.codebooks[:1]),
-        codes=idx.codes[:1].cpu().numpy(), list_ids=idx.list_ids[:1].cpu().numpy().view(np.uint16),
-        key_norms=f64(idx.key_norms[:1]), list_vmeans=f64(idx.list_vmeans[:1]),
-        k_cache_flat=f64(inp.k_cache[pages].reshape(-1)),
-        v_cache_flat=f64(inp.v_cache[pages].reshape(-1)),
-        block_table=np.arange(n_pages, dtype=np.int32)[None, :],
-        seq_lens=inp.seq_lens[:1].cpu().numpy())
+    """Float64 host copies of what the oracle needs for sequence 0 (index arrays and its own
+    KV pages); see tests/helpers.py."""
+    from helpers import oracle_arrays_for_sequence
+    return oracle_arrays_for_sequence(inp, idx, 0)
 
 
 def oracle_sample(inp, arrays, cfg, budget_ppm, n_heads):

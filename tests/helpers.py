@@ -30,6 +30,27 @@ def oracle_arrays(inp, idx):
     return a
 
 
+def oracle_arrays_for_sequence(inp, idx, b):
+    """Same as oracle_arrays, but for one sequence of a large workload: only that sequence's
+    index arrays and KV pages are copied to the host (pages re-packed contiguously with an
+    identity block table; the oracle still reads rows through block table and strides)."""
+    cfg = inp.cfg
+    assert cfg.kv_layout == "split"
+    f64 = lambda t: t.detach().cpu().double().numpy()
+    n = int(inp.seq_lens[b])
+    n_pages = max(1, (n + cfg.page_size - 1) // cfg.page_size)
+    pages = inp.block_table[b, :n_pages].long()
+    sl = slice(b, b + 1)
+    return dict(
+        q=f64(inp.q[sl]), centroids=f64(idx.centroids[sl]), codebooks=f64(idx.codebooks[sl]),
+        codes=idx.codes[sl].cpu().numpy(), list_ids=idx.list_ids[sl].cpu().numpy().view(np.uint16),
+        key_norms=f64(idx.key_norms[sl]), list_vmeans=f64(idx.list_vmeans[sl]),
+        k_cache_flat=f64(inp.k_cache[pages].reshape(-1)),
+        v_cache_flat=f64(inp.v_cache[pages].reshape(-1)),
+        block_table=np.arange(n_pages, dtype=np.int32)[None, :],
+        seq_lens=inp.seq_lens[sl].cpu().numpy())
+
+
 def run_oracle(inp, idx, budget_ppm=None, heads=None, batch_items=None, arrays=None):
     cfg = inp.cfg
     a = arrays or oracle_arrays(inp, idx)

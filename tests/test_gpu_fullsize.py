@@ -1,0 +1,68 @@
+"""Parity at the full sizes of the benchmark's configs, in the launch configuration bench.py times
+(-m gpu).  The oracle cannot redo every row of a 128K x 8-sequence batch in seconds, so each
+case checks sampled (sequence, query head) rows end to end: approximate logits over the whole
+row, the selected set, and the output."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_33746_b200 import pqhsa
+from paper_2609_33746_b200.index_builder import build_index
+from paper_2609_33746_b200.runner import DecodeOp
+from paper_2609_33746_b200.workload import generate, named_config
+
+from helpers import oracle_arrays_for_sequence, run_oracle, selection_matches
+from test_gpu_parity import LOGIT_RTOL, out_tolerance
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    # (workload, sampled (sequence, query head) rows)
+    ("c2", [(0, h) for h in (0, 5, 17, 31)]),
+    ("c3_b1_r1", [(0, 0), (0, 14), (0, 31)]),
+    ("c3_b1_r2", [(0, 9)]),
+    ("c3_b8_r1", [(0, 3), (4, 20), (7, 31)]),          # the benchmark's default workload
+    ("c4", [(2, 7), (11, 30)]),                        # ragged batch of 16, G = 8
+    ("c5_n512_b1", [(0, 1), (0, 30)]),                 # 512K context, n_list = 4096
+]
+
+
+@pytest.mark.parametrize("name,rows", CASES, ids=[c[0] for c in CASES])
+def test_full_size_decode_on_sampled_rows(name, rows):
+    cfg = dataclasses.replace(named_config(name), kmeans_iters=2)
+    inp = generate(cfg, device="cuda")
+    idx = build_index(inp)
+    op = DecodeOp(inp, idx)
+    out = op.decode()
+    torch.cuda.synchronize()
+    assert op.device_status() == pqhsa.OK
+    N_max, k_max = op.params.max_seq_len, op.params.k_max
+    scores = op.decode_buffer(pqhsa.BUF_SCORES).view(cfg.batch, cfg.n_q_heads, N_max)
+    sel = op.decode_buffer(pqhsa.BUF_SEL_IDX, torch.int32).view(cfg.batch, cfg.n_q_heads, k_max)
+    cnt = op.decode_buffer(pqhsa.BUF_SEL_COUNT, torch.int32).view(cfg.batch, cfg.n_q_heads)
+    by_seq = {}
+    for b, h in rows:
+        by_seq.setdefault(b, []).append(h)
+    for b, heads in by_seq.items():
+        arrays = oracle_arrays_for_sequence(inp, idx, b)
+        sub = dataclasses.replace(inp, cfg=dataclasses.replace(cfg, batch=1, seq_lens=(cfg.seq_lens[b],)))
+        ref = run_oracle(sub, None, heads=heads, batch_items=[0], arrays=arrays)
+        n = cfg.seq_lens[b]
+        for h in heads:
+            r = ref[(0, h)]
+            got = scores[b, h, :n].cpu().double().numpy()
+            assert np.all(np.abs(got - r["approx"]) <= LOGIT_RTOL * np.maximum(np.abs(r["approx"]), 1.0)), \
+                f"{name} logits row {(b, h)}: {np.abs(got - r['approx']).max()}"
+            c = int(cnt[b, h])
+            assert c == r["k"]
+            ok, why = selection_matches(sel[b, h, :c].cpu().numpy(), r)
+            assert ok, f"{name} selection row {(b, h)}: {why}"
+            y = out[b, h].cpu().double().numpy()
+            err = np.abs(y - r["y"])
+            assert np.all(err <= out_tolerance(r["y"], cfg.dtype)), \
+                f"{name} output row {(b, h)}: max-abs {err.max()}"
+    del op, inp, idx
+    torch.cuda.empty_cache()

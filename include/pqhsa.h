@@ -157,7 +157,7 @@ int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_p
  * For callers that cannot allocate device memory where they need the top-k: code running
  * inside an engine's pre-planned memory pool, plugins that receive tensors but no allocator,
  * and paths where a driver allocation -- which may stall the whole device -- is not
- * acceptable.  The scratch that pqhsa_select takes from `ws` (histograms, counters,
+ * acceptable.  The scratch that pqhsa_select takes from `ws` (counters and
  * candidate lists) lives instead in one fixed 16 MiB array inside the library image; every
  * GPU that loads the library holds that array until the process exits.
  *

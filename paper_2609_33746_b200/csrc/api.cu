@@ -87,7 +87,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.hist_chunks = ceil_div(4LL * o.num_sms, o.rows);
   if (o.hist_chunks > ceil_div(o.N_max, kSelChunk)) o.hist_chunks = ceil_div(o.N_max, kSelChunk);
   if (o.hist_chunks < 1) o.hist_chunks = 1;
-  o.cand_cap = o.N_max / 4 > 4096 ? o.N_max / 4 : 4096;
+  o.cand_cap = o.N_max / 4 > kSelChunk ? o.N_max / 4 : kSelChunk;
   if (o.cand_cap > o.N_max) o.cand_cap = o.N_max;
   // split-K CTAs per row: about 256 selected tokens each, but enough CTAs to fill the GPU
   // when there are few rows, as long as every CTA keeps at least 32 units of work
@@ -123,8 +123,6 @@ void make_layout(const Plan& pl, WsLayout* L) {
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
   L->zero_begin = o;
   L->status = take(16);
-  L->hist1 = take((size_t)pl.rows * kHistBins * 4);
-  L->hist2 = take((size_t)pl.rows * kHistBins * 4);
   L->counters = take((size_t)pl.rows * 16);
   L->attend_tickets = take((size_t)pl.rows * 4);
   L->bg_mass = take((size_t)pl.rows * pl.n_list * 4);
@@ -232,7 +230,7 @@ int pqhsa_decode_launch_count(const pqhsa_params* params) {
   Plan pl;
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
-  return 6;   // LUT build, scan, select histogram, select filter, background prep, attend
+  return 6;   // LUT build, scan, select sample, select filter, background prep, attend
 }
 
 int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index* index,

@@ -19,7 +19,7 @@ constexpr int kTile = 32;            // tokens per scan tile: one token per lane
 #endif
 constexpr int kScanThreads = PQHSA_SCAN_THREADS;
 constexpr int kScanMinTiles = kScanThreads / 32;   // a scan CTA gets at least one tile per warp
-constexpr int kHistBins = 4096;      // 12-bit radix digits for the two coarse select levels
+constexpr int kHistBins = 4096;      // 12-bit radix digits of the select's shared-memory histograms
 constexpr int kSelThreads = 512;
 constexpr int kSelChunk = 8192;      // scores per select CTA: 16 per thread, kept in registers
 constexpr int kAttendThreads = 128;
@@ -52,11 +52,10 @@ struct Plan {
 struct WsLayout {
   size_t status;                     // int32[4]: device status word (+ padding)
   size_t zero_begin, zero_bytes;     // region cleared by one memset before select
-  size_t hist1, hist2;               // uint32 [rows][kHistBins] each
-  size_t counters;                   // uint32 [rows][4]: ticket1, ticket2, n_out, n_cand
+  size_t counters;                   // uint32 [rows][4]: fallbacks, ticket, n_out, n_cand
   size_t attend_tickets;             // uint32 [rows]
   size_t attend_zero_bytes;          // tickets + bg_mass: what the attend stage needs cleared
-  size_t rowstate;                   // int32  [rows][4]: b1, k1, k, n
+  size_t rowstate;                   // int32  [rows][4]: lo, hi (float bits), k, n
   size_t cand;                       // uint2  [rows][cand_cap]: (key, position)
   size_t bg_mass;                    // float  [rows][n_list]: M_j relative to bg_max (accumulated)
   size_t bg_max;                     // float  [rows]

@@ -4,7 +4,7 @@
 // code that runs inside an engine's already-planned memory pool, plugins that are handed
 // tensors but no allocator, and latency-critical paths where a driver allocation (which may
 // synchronise the whole device) is not acceptable.  pqhsa_select needs a caller-provided
-// workspace for its histograms, counters and candidate lists; this variant keeps that scratch
+// workspace for its counters and candidate lists; this variant keeps that scratch
 // in one fixed array that is part of the library image, so the caller passes only inputs and
 // outputs.  The price: a fixed upper size, and one array shared by every call on a device.
 #include <mutex>
@@ -45,15 +45,13 @@ cudaError_t scratch_address(unsigned char** out) {
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 // Only what the top-k kernels touch, packed from offset 0; the first `zero_bytes` bytes are
-// the part that must start at zero (status word, histograms, counters).
+// the part that must start at zero (status word, counters).
 void make_select_layout(const Plan& pl, WsLayout* L) {
   *L = WsLayout{};
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
   L->zero_begin = 0;
   L->status = take(16);
-  L->hist1 = take((size_t)pl.rows * kHistBins * 4);
-  L->hist2 = take((size_t)pl.rows * kHistBins * 4);
   L->counters = take((size_t)pl.rows * 16);
   L->zero_bytes = o;
   L->rowstate = take((size_t)pl.rows * 16);

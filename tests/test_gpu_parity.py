@@ -232,17 +232,16 @@ def test_selection_is_deterministic_and_stable_on_ties():
             assert sorted(r[h, :k].tolist()) == want.tolist()
 
 
-def test_candidate_overflow_path():
-    """More candidates in the threshold digit than the candidate buffer holds: the last CTA
-    falls back to re-reading the score row."""
-    cfg = small("overflow", seq_lens=(32768,), n_q_heads=4, n_kv_heads=1, budget_ppm=500000,
+def test_many_candidates_take_the_global_list_path():
+    """Half of the row is selected from a narrow range of scores: the bracket holds more
+    candidates than fit in shared memory, so the last CTA works from the global list."""
+    cfg = small("wide", seq_lens=(32768,), n_q_heads=4, n_kv_heads=1, budget_ppm=500000,
                 kmeans_iters=1, n_list=16)
     inp, idx = make_case(cfg, device="cuda")
     op = DecodeOp(inp, idx)
     op.alloc_stage_buffers()
     N = op.params.max_seq_len
     g = torch.Generator(device="cuda").manual_seed(5)
-    # all scores inside one top-level digit (same sign / exponent / top mantissa bits)
     sc = 1.0 + torch.rand((4, N), generator=g, device="cuda") * 0.05
     op.scores.view(1, 4, N)[0] = sc
     op.select()
@@ -253,6 +252,43 @@ def test_candidate_overflow_path():
     for h in range(4):
         want = O.select_topk(sc[h].cpu().double().numpy(), k)
         assert sorted(got[h, :k].tolist()) == want.tolist()
+
+
+def sampled_positions(n, n_sample=4096):
+    """The positions the select's sample kernel reads in a row of n scores."""
+    i = np.arange(n_sample, dtype=np.int64)
+    a, z = i * n // n_sample, (i + 1) * n // n_sample
+    h = (i * 2654435761) & 0xFFFFFFFF
+    return a + (h >> 8) % (z - a)
+
+
+def test_rows_that_defeat_the_sample_fall_back_to_the_exact_path():
+    """All of the top-k scores sit where the sample does not look, so the sample's bracket
+    misses; the count check catches it and the last CTA selects from the row itself.  Also:
+    ascending and descending rows (top-k in one corner) and a row with one huge outlier."""
+    cfg = small("defeat", seq_lens=(65536,), n_q_heads=4, n_kv_heads=1, budget_ppm=10000,
+                kmeans_iters=1, n_list=16)
+    inp, idx = make_case(cfg, device="cuda")
+    op = DecodeOp(inp, idx)
+    op.alloc_stage_buffers()
+    N = op.params.max_seq_len
+    k = O.budget_k(N, 10000)
+    g = torch.Generator(device="cuda").manual_seed(9)
+    sc = torch.randn((4, N), generator=g, device="cuda")
+    hidden = np.setdiff1d(np.arange(N), sampled_positions(N))[:k]
+    sc[0, torch.from_numpy(hidden).cuda()] += 100.0          # top-k invisible to the sample
+    sc[1] = torch.arange(N, device="cuda", dtype=torch.float32) * 1e-3
+    sc[2] = -torch.arange(N, device="cuda", dtype=torch.float32) * 1e-3
+    sc[3, 12345] = 1e30
+    op.scores.view(1, 4, N)[0] = sc
+    op.select()
+    torch.cuda.synchronize()
+    assert op.device_status() == pqhsa.OK
+    got = op.sel_idx.view(4, -1).cpu().numpy()
+    for h in range(4):
+        want = O.select_topk(sc[h].cpu().double().numpy(), k)
+        assert sorted(got[h, :k].tolist()) == want.tolist()
+    assert sorted(got[0, :k].tolist()) == sorted(hidden.tolist())
 
 
 def test_invalid_arguments_launch_nothing():

@@ -34,6 +34,8 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   const int b = row / pl.Hq, h = row % pl.Hq;
   const int kv = h / pl.G, hg = (h % pl.G) / pl.Gc;
   const int n_list = pl.n_list;
+  pdl_wait();
+  pdl_launch_dependents();
   const int n = clamp_len(seq_lens[b], pl.N_max);
   float* mass = bg_mass + (size_t)row * n_list;
   if (n == 0) {
@@ -166,6 +168,8 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   const int b = row / pl.Hq, h = row % pl.Hq, kv = h / pl.G;
   const size_t ukv = (size_t)b * pl.Hkv + kv;
   const int n_list = pl.n_list;
+  pdl_wait();
+  pdl_launch_dependents();
   const int cnt = sel_count[row];
 
   // ---- this warp's slice of the selected tokens: resolve cache offsets first (two
@@ -388,24 +392,25 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
   float* bg_max = reinterpret_cast<float*>(ws + L.bg_max);
   float* split_part = reinterpret_cast<float*>(ws + L.split_part);
   uint32_t* tickets = reinterpret_cast<uint32_t*>(ws + L.attend_tickets);
-  bg_prep_kernel<<<dim3(pl.bg_ctas, pl.rows), kBgThreads, 0, st>>>(
-      pl, scores, list_partials, sel_idx, sel_count, ix.list_ids, seq_lens, bg_mass, bg_max);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_pdl(bg_prep_kernel, dim3(pl.bg_ctas, pl.rows), dim3(kBgThreads), 0, st, pl,
+                             scores, list_partials, sel_idx, sel_count, ix.list_ids, seq_lens,
+                             bg_mass, bg_max);
   if (e != cudaSuccess) return e;
   dim3 grid(pl.splits, pl.rows);
   if (pl.dtype == PQHSA_F16)
-    attend_kernel<__half, 4><<<grid, kAttendThreads, 0, st>>>(
-        pl, static_cast<const __half*>(q), static_cast<const __half*>(kv.k_cache),
-        static_cast<const __half*>(kv.v_cache), kv.stride_page, kv.stride_token, kv.stride_head,
-        kv.block_table, sel_idx, sel_count, bg_mass, bg_max, ix.list_vmeans, split_part, tickets,
-        static_cast<__half*>(out), lse);
-  else
-    attend_kernel<__nv_bfloat16, 4><<<grid, kAttendThreads, 0, st>>>(
-        pl, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kv.k_cache),
-        static_cast<const __nv_bfloat16*>(kv.v_cache), kv.stride_page, kv.stride_token,
-        kv.stride_head, kv.block_table, sel_idx, sel_count, bg_mass, bg_max, ix.list_vmeans,
-        split_part, tickets, static_cast<__nv_bfloat16*>(out), lse);
-  return cudaGetLastError();
+    return launch_pdl(attend_kernel<__half, 4>, grid, dim3(kAttendThreads), 0, st, pl,
+                      static_cast<const __half*>(q), static_cast<const __half*>(kv.k_cache),
+                      static_cast<const __half*>(kv.v_cache), (long long)kv.stride_page,
+                      (long long)kv.stride_token, (long long)kv.stride_head, kv.block_table,
+                      sel_idx, sel_count, bg_mass, bg_max, ix.list_vmeans, split_part, tickets,
+                      static_cast<__half*>(out), lse);
+  return launch_pdl(attend_kernel<__nv_bfloat16, 4>, grid, dim3(kAttendThreads), 0, st, pl,
+                    static_cast<const __nv_bfloat16*>(q),
+                    static_cast<const __nv_bfloat16*>(kv.k_cache),
+                    static_cast<const __nv_bfloat16*>(kv.v_cache), (long long)kv.stride_page,
+                    (long long)kv.stride_token, (long long)kv.stride_head, kv.block_table, sel_idx,
+                    sel_count, bg_mass, bg_max, ix.list_vmeans, split_part, tickets,
+                    static_cast<__nv_bfloat16*>(out), lse);
 }
 
 }  // namespace pqhsa

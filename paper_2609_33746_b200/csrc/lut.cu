@@ -54,6 +54,8 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
   const int G = pl.G, Gc = pl.Gc, n_hg = pl.n_hg;
   const int n_slots = n_hg * Gc;                            // head slots, >= G
   const size_t ukv = (size_t)b * pl.Hkv + kv;
+  pdl_wait();
+  pdl_launch_dependents();
 
   // query (first dependent load of the kernel)
   float qreg[(kMaxGroup * kHeadDim) / kLutThreads];
@@ -176,10 +178,10 @@ static cudaError_t launch_lut_t(const Plan& pl, const T* q, const pqhsa_index& i
                                 float* coarse, uint4* zp, size_t zn, cudaStream_t st) {
   dim3 grid(kLutChunks, pl.Hkv, pl.B);
   switch (pl.dsub) {
-    case 2: build_lut_kernel<T, 2><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
-    case 4: build_lut_kernel<T, 4><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
-    case 8: build_lut_kernel<T, 8><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
-    case 16: build_lut_kernel<T, 16><<<grid, kLutThreads, 0, st>>>(pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn); break;
+    case 2: return launch_pdl(build_lut_kernel<T, 2>, grid, dim3(kLutThreads), 0, st, pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn);
+    case 4: return launch_pdl(build_lut_kernel<T, 4>, grid, dim3(kLutThreads), 0, st, pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn);
+    case 8: return launch_pdl(build_lut_kernel<T, 8>, grid, dim3(kLutThreads), 0, st, pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn);
+    case 16: return launch_pdl(build_lut_kernel<T, 16>, grid, dim3(kLutThreads), 0, st, pl, q, ix.centroids, ix.codebooks, lut, coarse, zp, zn);
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();

@@ -222,6 +222,8 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   const int c = blockIdx.x;
   const int n_list = pl.n_list, N_max = pl.N_max, upb = pl.upb;
 
+  pdl_wait();
+  pdl_launch_dependents();
   const ScanSplit sp = scan_split(seq_lens, pl.B, N_max, upb, pl.scan_ctas);
   if (c == 0 && tid == 0) {
     for (int b = 0; b < pl.B; ++b)
@@ -472,9 +474,9 @@ static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const fl
   cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  scan_kernel<M, GC, S><<<pl.scan_ctas, kScanThreads, smem, st>>>(
-      pl, ix.codes, ix.list_ids, ix.key_norms, lut, coarse, seq_lens, scores, partials, status);
-  return cudaGetLastError();
+  return launch_pdl(scan_kernel<M, GC, S>, dim3(pl.scan_ctas), dim3(kScanThreads), smem, st, pl,
+                    ix.codes, ix.list_ids, ix.key_norms, lut, coarse, seq_lens, scores, partials,
+                    status);
 }
 
 cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,

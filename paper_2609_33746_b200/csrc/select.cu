@@ -2,7 +2,7 @@
 // T(q) = TopK_{k, i in R} l~_i with k = ceil(rho |R|).
 //
 // One pass over the scores instead of a multi-pass radix sort of the whole row:
-//   sample kernel  one CTA per row reads 4096 scores spread over the row (jittered stride)
+//   sample kernel  one CTA per row reads 4096 scores (1024 groups of 4, jittered stride)
 //                  and takes two order statistics of the sample that bracket the k-th largest
 //                  score of the row with a 6-sigma margin: lo <= s_k <= hi;
 //   filter kernel  scores above hi are certain winners and are written out at once; scores in
@@ -24,6 +24,7 @@ constexpr int kElems = kSelChunk / kSelThreads;   // scores per thread per chunk
 constexpr int kStashCap = 3072;                   // candidates resolved from shared memory
 constexpr int kSample = 4096;                     // sampled scores per row
 constexpr int kSamplePer = kSample / kSelThreads; // per thread (8)
+constexpr int kSampleGroups = kSample / 4;        // groups of 4 consecutive scores
 constexpr float kBracketSigmas = 6.0f;
 
 // rowstate: [0] lo, [1] hi (float bits), [2] k, [3] n
@@ -169,6 +170,8 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
   __shared__ int s_scan[34];
   const int row = blockIdx.x, tid = threadIdx.x;
   const int b = row / pl.Hq;
+  pdl_wait();
+  pdl_launch_dependents();
   const int n = clamp_len(seq_lens[b], pl.N_max);
   const int k = budget_k(n, pl.ppm);
   float lo = -CUDART_INF_F, hi = CUDART_INF_F;     // default: every score is a candidate
@@ -177,15 +180,19 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
   } else if (k == n) {
     hi = -CUDART_INF_F;                            // every finite score is a winner
   } else if (n > kSelChunk) {
-    // sample i sits in the i-th of 4096 equal strides of the row, at a hashed offset
+    // 1024 aligned groups of 4 consecutive scores; group g sits in the g-th of 1024 equal
+    // strides of the row at a hashed offset (reads 16 bytes per touched 32-byte sector)
     const float* rs = scores + (size_t)row * pl.N_max;
     float s[kSamplePer];
 #pragma unroll
-    for (int e = 0; e < kSamplePer; ++e) {
-      const int i = e * kSelThreads + tid;
-      const long long a = (long long)i * n / kSample, z = (long long)(i + 1) * n / kSample;
-      const uint32_t h = (uint32_t)i * 2654435761u;
-      s[e] = __ldcg(rs + a + (long long)((h >> 8) % (uint32_t)(z - a)));
+    for (int u = 0; u < kSamplePer / 4; ++u) {
+      const int g = u * kSelThreads + tid;
+      const long long a = (long long)g * n / kSampleGroups, z = (long long)(g + 1) * n / kSampleGroups;
+      const uint32_t h = (uint32_t)g * 2654435761u;
+      long long off = (a + (long long)((h >> 8) % (uint32_t)(z - a))) & ~3LL;
+      if (off + 4 > n) off = (n - 4) & ~3LL;
+      const float4 f = __ldcg(reinterpret_cast<const float4*>(rs + off));
+      s[4 * u] = f.x; s[4 * u + 1] = f.y; s[4 * u + 2] = f.z; s[4 * u + 3] = f.w;
     }
     uint32_t key[kSamplePer];
 #pragma unroll
@@ -336,6 +343,8 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
   __shared__ uint32_t s_emit;
   const int row = blockIdx.y, tid = threadIdx.x, chunk = blockIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
+  pdl_wait();
+  pdl_launch_dependents();
   const float lo_f = __int_as_float(rowstate[row * 4 + 0]);
   const float hi_f = __int_as_float(rowstate[row * 4 + 1]);
   const int k = rowstate[row * 4 + 2], n = rowstate[row * 4 + 3];
@@ -465,13 +474,11 @@ cudaError_t launch_select(const Plan& pl, const WsLayout& L, char* ws, const flo
   int32_t* rowstate = reinterpret_cast<int32_t*>(ws + L.rowstate);
   uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
   int* status = reinterpret_cast<int*>(ws + L.status);
-  sel_sample_kernel<<<pl.rows, kSelThreads, 0, st>>>(pl, scores, seq_lens, rowstate, sel_count,
-                                                     kth);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_pdl(sel_sample_kernel, dim3(pl.rows), dim3(kSelThreads), 0, st, pl, scores,
+                             seq_lens, rowstate, sel_count, kth);
   if (e != cudaSuccess) return e;
-  sel_filter_kernel<<<dim3(pl.hist_chunks, pl.rows), kSelThreads, 0, st>>>(
-      pl, scores, counters, rowstate, cand, sel_idx, sel_count, kth, status);
-  return cudaGetLastError();
+  return launch_pdl(sel_filter_kernel, dim3(pl.hist_chunks, pl.rows), dim3(kSelThreads), 0, st, pl,
+                    scores, counters, rowstate, cand, sel_idx, sel_count, kth, status);
 }
 
 }  // namespace pqhsa

@@ -254,12 +254,14 @@ def test_many_candidates_take_the_global_list_path():
         assert sorted(got[h, :k].tolist()) == want.tolist()
 
 
-def sampled_positions(n, n_sample=4096):
-    """The positions the select's sample kernel reads in a row of n scores."""
-    i = np.arange(n_sample, dtype=np.int64)
-    a, z = i * n // n_sample, (i + 1) * n // n_sample
-    h = (i * 2654435761) & 0xFFFFFFFF
-    return a + (h >> 8) % (z - a)
+def sampled_positions(n, n_groups=1024):
+    """The positions the select's sample kernel reads in a row of n scores (1024 groups of 4)."""
+    g = np.arange(n_groups, dtype=np.int64)
+    a, z = g * n // n_groups, (g + 1) * n // n_groups
+    h = (g * 2654435761) & 0xFFFFFFFF
+    off = (a + (h >> 8) % (z - a)) & ~3
+    off = np.where(off + 4 > n, (n - 4) & ~3, off)
+    return (off[:, None] + np.arange(4)[None, :]).ravel()
 
 
 def test_rows_that_defeat_the_sample_fall_back_to_the_exact_path():

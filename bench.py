@@ -32,6 +32,7 @@ METRIC = ("decode-attention achieved HBM GB/s at 128K context "
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 512 << 20
+SCAN_DRAM_BYTES_PER_UNIT = 41.15e6 / (8 * 131072)   # ncu, profiles/scan_kernel_c3_b1.md
 
 
 def measured_peak():
@@ -306,8 +307,8 @@ def main():
     assert op.device_status() == pqhsa.OK
 
     sampler.start()
+    time.sleep(0.3)                      # let nvidia-smi come up before the first timed step
     head = measure(op, cfg, cfg.budget_ppm, args.steps, args.warmup, seq_lens)
-    clocks = sampler.stop()
     launches = args.steps * pqhsa.decode_launch_count(op.params)
 
     # per-stage times of the same call, recorded by the library around its own stages
@@ -316,9 +317,18 @@ def main():
     peak, peak_src = measured_peak()
     scan_bytes = head["bytes"]["scan"]
     scan_gbs = scan_bytes / (stage_ms[1] * 1e-3) / 1e9
+    # DRAM bytes of one scan launch: ncu counted 41.15 MB for the 8 x 131072 tokens of
+    # c3_b1 (profiles/scan_kernel_c3_b1.md) = 39.2 B per (token, KV head), scaled by units
+    scan_units = cfg.n_kv_heads * sum(seq_lens)
+    scan_traffic = SCAN_DRAM_BYTES_PER_UNIT * scan_units
     roofline = dict(bound="hbm", kernel="scan_kernel (ADC scan + fused per-list sums)",
                     achieved=scan_gbs, peak=peak, unit="GB/s", frac=scan_gbs / peak,
-                    peak_source=peak_src, traffic=None,
+                    peak_source=peak_src, traffic=scan_traffic,
+                    traffic_note="dram__bytes_read+write of one ncu capture on c3_b1, scaled by "
+                                 "tokens x KV heads; score rows written by the scan stay in L2 "
+                                 "past the end of the kernel, so they are not in this figure",
+                    binding_unit="shared-memory LSU (l1tex data-pipe wavefronts), not HBM: "
+                                 "see profiles/scan_kernel_c3_b1.md",
                     algorithmic_bytes_per_launch=scan_bytes, avg_launch_ms=stage_ms[1],
                     co_bound="shared-memory LSU: 16 B of table reads per (token, subspace)",
                     stage_ms=dict(lut=stage_ms[0], scan=stage_ms[1], select=stage_ms[2],
@@ -365,6 +375,7 @@ def main():
                 algorithmic_mb=r["bytes"]["total"] / 1e6)
             del op_v
 
+    clocks = sampler.stop()              # sampled over every timed loop above
     cpu_baseline = None
     if rank == 0 and world == 1:
         heads = max(1, min(args.oracle_heads, cfg.n_q_heads))

@@ -82,9 +82,11 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   else if (scan_smem_bytes(o, false, 2) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 2; }
   else return PQHSA_ERR_UNSUPPORTED;
 
-  // select CTAs per row: enough CTAs to fill the GPU about twice over, each looping over
-  // 8192-score chunks of its row
-  o.hist_chunks = ceil_div(4LL * o.num_sms, o.rows);
+  // select CTAs per row, each looping over 8192-score chunks of its row: with few rows
+  // exactly one wave of resident CTAs (3 per SM; a straggling second wave would double the
+  // kernel), with many rows short CTAs in at least two waves
+  const int sel_slots = 3 * o.num_sms;
+  o.hist_chunks = 2 * o.rows <= sel_slots ? sel_slots / o.rows : ceil_div(2LL * sel_slots, o.rows);
   if (o.hist_chunks > ceil_div(o.N_max, kSelChunk)) o.hist_chunks = ceil_div(o.N_max, kSelChunk);
   if (o.hist_chunks < 1) o.hist_chunks = 1;
   o.cand_cap = o.N_max / 4 > kSelChunk ? o.N_max / 4 : kSelChunk;
@@ -92,7 +94,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   // split-K CTAs per row: about 256 selected tokens each, but enough CTAs to fill the GPU
   // when there are few rows, as long as every CTA keeps at least 32 units of work
   o.splits = ceil_div(o.k_max, 256);
-  int fill = ceil_div(4LL * o.num_sms, o.rows);
+  int fill = (4 * o.num_sms) / o.rows;     // one wave of resident CTAs (4 per SM)
   const int max_fill = (o.k_max + o.n_list / 4) / 32 > 0 ? (o.k_max + o.n_list / 4) / 32 : 1;
   if (fill > max_fill) fill = max_fill;
   if (o.splits < fill) o.splits = fill;

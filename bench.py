@@ -160,8 +160,8 @@ def parse_workload(name):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="c3_b8_r1",
                     help="c3_b{1,8}_r{1,2} (128K, headline), c2, c4, c5_n{16..512}_b{1,32}")
     ap.add_argument("--impl", default="pqhsa", choices=["pqhsa", "reference"])
@@ -375,6 +375,48 @@ def main():
                 algorithmic_mb=r["bytes"]["total"] / 1e6)
             del op_v
 
+    # dense comparator: the library's own split-K dense decode kernel over the same paged cache
+    dws = torch.empty(pqhsa.dense_workspace_bytes(op.params), dtype=torch.uint8, device=dev)
+    dout = torch.empty_like(op.q)
+    for _ in range(3):
+        pqhsa.dense_decode(op.params, op.q, op.kv, op.seq_lens, dout, dws)
+    dsteps = max(5, args.steps // 4)
+    dev_pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                 for _ in range(dsteps)]
+    barrier()
+    for a, b in dev_pairs:
+        flush.zero_()
+        a.record()
+        pqhsa.dense_decode(op.params, op.q, op.kv, op.seq_lens, dout, dws)
+        b.record()
+    barrier()
+    dense_ms = reduce_max(sum(a.elapsed_time(b) for a, b in dev_pairs) / dsteps)
+    dbytes = dense_attention_bytes(cfg, seq_lens)
+    dense = dict(us_per_step=1000 * dense_ms, achieved_gbs=dbytes / (dense_ms * 1e-3) / 1e9,
+                 bytes=dbytes, speedup_over_dense=dense_ms / head["ms"],
+                 kernel="dense_decode_kernel (own split-K dense decode attention, same cache)")
+
+    # the same step replayed from a CUDA graph (no per-launch host work)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        op.decode()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        op.decode()
+    g_pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+    barrier()
+    for a, b in g_pairs:
+        flush.zero_()
+        a.record()
+        graph.replay()
+        b.record()
+    barrier()
+    graph_ms = reduce_max(sum(a.elapsed_time(b) for a, b in g_pairs) / len(g_pairs))
+
     clocks = sampler.stop()              # sampled over every timed loop above
     cpu_baseline = None
     if rank == 0 and world == 1:
@@ -407,7 +449,8 @@ def main():
             key_tokens_scanned_per_s=world * cfg.n_kv_heads * n_tok / (head["ms"] * 1e-3),
             algorithmic_bytes_per_step=head["bytes"], dense_attention_bytes=dense_attention_bytes(cfg, seq_lens),
             clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roofline,
-            cpu_baseline=cpu_baseline, variants=variants,
+            cpu_baseline=cpu_baseline, variants=variants, dense_comparator=dense,
+            graph_replay_us_per_step=1000 * graph_ms,
             context_only="paper: 1.58x over FlashAttention-3 on one H20 at 128K, 1% (other "
                          "hardware, other index setting)")
         print(json.dumps(line))

@@ -193,6 +193,16 @@ int pqhsa_decode_events(const pqhsa_params* params, const void* q, const pqhsa_i
                         const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out,
                         void* ws, size_t ws_bytes, void* stream, void* const* stage_events);
 
+/* Dense decode attention over the WHOLE paged KV cache (Eq. 1 with E = every cached token):
+ * softmax(q K^T / sqrt d) V per query head, split-K with a log-sum-exp merge.  Not a step of
+ * PQ-HSA: it is the comparator of the context-length sweep (the full-KV read the paper's
+ * Sec. 4.4 measures against), run on the same cache through the same strides.  Uses batch,
+ * heads, head_dim, max_seq_len, page fields, sm_scale and dtype of `params`.  `ws`: device
+ * scratch of pqhsa_dense_workspace_bytes(params) bytes, 256-byte aligned. */
+size_t pqhsa_dense_workspace_bytes(const pqhsa_params* params);
+int pqhsa_dense_decode(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
+                       const int32_t* seq_lens, void* out, void* ws, size_t ws_bytes, void* stream);
+
 /* pqhsa_decode for a caller whose query and output live in HOST memory (pinned for the
  * copies to be asynchronous): copies q_host -> q_dev_staging, runs the step, copies
  * out_dev_staging -> out_host and waits for the stream.  The index, the KV cache and

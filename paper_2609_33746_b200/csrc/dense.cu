@@ -1,0 +1,225 @@
+// Dense decode attention over the whole paged KV cache: the comparator of the context-length
+// sweep (Eq. 1 with E = every cached token).  Not part of the PQ-HSA path; it exists so that
+// the operator's time can be set against a full-KV read on the same GPU and the same cache.
+//
+// Split-K flash decoding.  grid (splits, KV heads, sequences); the CTA has one warp per query
+// head of the GQA group, and all warps walk the same slice of tokens, so a K/V row comes from
+// HBM once and from L1 for the other heads.  Inside a warp: 8 lanes per 256-byte row, 16 rows
+// in flight, online softmax in base 2.  The last CTA of a (sequence, KV head) merges the
+// partial (m, Z, N) triples of its G rows (atomic ticket; nobody waits).
+#include "attn_common.cuh"
+#include "common.cuh"
+
+namespace pqhsa {
+
+namespace {
+
+constexpr int kDensePart = 2 + kHeadDim;
+constexpr int kMaxDenseWarps = 16;
+
+template <typename T, int U>
+__global__ void __launch_bounds__(32 * kMaxDenseWarps)
+dense_decode_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc,
+                    const T* __restrict__ vc, long long stride_page, long long stride_token,
+                    long long stride_head, const int32_t* __restrict__ block_table,
+                    const int32_t* __restrict__ seq_lens, float* __restrict__ part,
+                    uint32_t* __restrict__ tickets, T* __restrict__ out) {
+  __shared__ int s_last;
+  const int split = blockIdx.x, S = gridDim.x, kv = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row = b * pl.Hq + kv * pl.G + warp;         // one query head per warp
+  pdl_wait();
+  pdl_launch_dependents();
+  const int n = clamp_len(seq_lens[b], pl.N_max);
+  const int tl = (int)((long long)split * n / S), th = (int)((long long)(split + 1) * n / S);
+  const int32_t* bt = block_table + (size_t)b * pl.max_pages;
+
+  const int gi = lane >> 3, gl = lane & 7;
+  float qf[16];
+  {
+    const T* qr = q + (size_t)row * kHeadDim;
+    const float sc = pl.sm_scale * kLog2e;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      qf[t] = sc * Unpack<T>::one(qr[8 * gl + t]);
+      qf[8 + t] = sc * Unpack<T>::one(qr[64 + 8 * gl + t]);
+    }
+  }
+  GroupState st;
+  st.m = -CUDART_INF_F;
+  st.Z = 0.f;
+#pragma unroll
+  for (int t = 0; t < 16; ++t) st.acc[t] = 0.f;
+
+  int my_page = (tl + lane < th) ? __ldg(bt + (tl + lane) / pl.page_size) : 0;
+  for (int base = tl; base < th; base += 32) {
+    const int pos = base + lane;
+    long long off = 0;
+    if (pos < th)
+      off = (long long)my_page * stride_page + (long long)(pos % pl.page_size) * stride_token +
+            (long long)kv * stride_head;
+    const int nb = min(32, th - base);
+    for (int j0 = 0; j0 < nb; j0 += 4 * U) {
+      uint4 kr[U][2], vr[U][2];
+      bool ok[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int tok = j0 + 4 * u + gi;
+        const long long o = __shfl_sync(0xffffffffu, off, tok & 31);
+        ok[u] = tok < nb;
+        if (ok[u]) {
+          const uint4* kp = reinterpret_cast<const uint4*>(kc + o);
+          const uint4* vp = reinterpret_cast<const uint4*>(vc + o);
+          kr[u][0] = __ldg(kp + gl); kr[u][1] = __ldg(kp + 8 + gl);
+          vr[u][0] = __ldg(vp + gl); vr[u][1] = __ldg(vp + 8 + gl);
+        } else {
+          kr[u][0] = kr[u][1] = vr[u][0] = vr[u][1] = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+      if (j0 == 0 && base + 32 + lane < th) my_page = __ldg(bt + (base + 32 + lane) / pl.page_size);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float kf[8];
+        float s = 0.f;
+        Unpack<T>::run(kr[u][0], kf);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) s = fmaf(qf[t], kf[t], s);
+        Unpack<T>::run(kr[u][1], kf);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) s = fmaf(qf[8 + t], kf[t], s);
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        s += __shfl_xor_sync(0xffffffffu, s, 4);
+        if (ok[u]) {
+          if (s > st.m) {
+            const float a = st.Z > 0.f ? fast_exp2(st.m - s) : 0.f;
+            st.Z *= a;
+#pragma unroll
+            for (int t = 0; t < 16; ++t) st.acc[t] *= a;
+            st.m = s;
+          }
+          const float p = fast_exp2(s - st.m);
+          st.Z += p;
+          float vf[8];
+          Unpack<T>::run(vr[u][0], vf);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) st.acc[t] = fmaf(p, vf[t], st.acc[t]);
+          Unpack<T>::run(vr[u][1], vf);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) st.acc[8 + t] = fmaf(p, vf[t], st.acc[8 + t]);
+        }
+      }
+    }
+  }
+  // merge the 4 lane groups of the warp
+#pragma unroll
+  for (int o = 8; o <= 16; o <<= 1) {
+    const float m_o = __shfl_xor_sync(0xffffffffu, st.m, o);
+    const float Z_o = __shfl_xor_sync(0xffffffffu, st.Z, o);
+    const float m_n = fmaxf(st.m, m_o);
+    const float a = safe_scale(st.m, m_n, st.Z), bsc = safe_scale(m_o, m_n, Z_o);
+    st.Z = st.Z * a + Z_o * bsc;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      const float acc_o = __shfl_xor_sync(0xffffffffu, st.acc[t], o);
+      st.acc[t] = st.acc[t] * a + acc_o * bsc;
+    }
+    st.m = m_n;
+  }
+  float* pr = part + ((size_t)row * S + split) * kDensePart;
+  if (gi == 0) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      pr[2 + 8 * gl + t] = st.acc[t];
+      pr[2 + 64 + 8 * gl + t] = st.acc[8 + t];
+    }
+    if (gl == 0) { pr[0] = st.m; pr[1] = st.Z; }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&tickets[b * pl.Hkv + kv], 1u) == (uint32_t)(S - 1));
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // last CTA of this (sequence, KV head): each warp merges its row; a lane owns 4 dims
+  const float* rp = part + (size_t)row * S * kDensePart;
+  float m_r = -CUDART_INF_F;
+  for (int s = 0; s < S; ++s)
+    if (__ldcg(rp + s * kDensePart + 1) > 0.f) m_r = fmaxf(m_r, __ldcg(rp + s * kDensePart));
+  float Z_r = 0.f;
+  float4 N_r = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < S; ++s) {
+    const float Zs = __ldcg(rp + s * kDensePart + 1);
+    const float a = safe_scale(__ldcg(rp + s * kDensePart), m_r, Zs);
+    const float* np = rp + s * kDensePart + 2 + 4 * lane;
+    Z_r = fmaf(Zs, a, Z_r);
+    N_r.x = fmaf(__ldcg(np), a, N_r.x); N_r.y = fmaf(__ldcg(np + 1), a, N_r.y);
+    N_r.z = fmaf(__ldcg(np + 2), a, N_r.z); N_r.w = fmaf(__ldcg(np + 3), a, N_r.w);
+  }
+  const float inv = Z_r > 0.f ? 1.f / Z_r : 0.f;
+  T* o = out + (size_t)row * kHeadDim + 4 * lane;
+  o[0] = Unpack<T>::pack(N_r.x * inv); o[1] = Unpack<T>::pack(N_r.y * inv);
+  o[2] = Unpack<T>::pack(N_r.z * inv); o[3] = Unpack<T>::pack(N_r.w * inv);
+}
+
+int dense_splits(const Plan& pl) {
+  int s = (4 * pl.num_sms) / (pl.B * pl.Hkv);
+  const int max_s = pl.N_max / 256 > 0 ? pl.N_max / 256 : 1;
+  if (s > max_s) s = max_s;
+  if (s > 256) s = 256;
+  return s < 1 ? 1 : s;
+}
+
+size_t align256d(size_t x) { return (x + 255) / 256 * 256; }
+
+}  // namespace
+}  // namespace pqhsa
+
+using namespace pqhsa;
+
+extern "C" {
+
+size_t pqhsa_dense_workspace_bytes(const pqhsa_params* params) {
+  Plan pl;
+  if (make_plan(params, &pl) != PQHSA_OK) return 0;
+  return align256d((size_t)pl.B * pl.Hkv * 4) +
+         align256d((size_t)pl.rows * dense_splits(pl) * kDensePart * 4);
+}
+
+int pqhsa_dense_decode(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
+                       const int32_t* seq_lens, void* out, void* ws, size_t ws_bytes, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if (q == nullptr || kv == nullptr || kv->k_cache == nullptr || kv->v_cache == nullptr ||
+      kv->block_table == nullptr || seq_lens == nullptr || out == nullptr || ws == nullptr ||
+      (reinterpret_cast<uintptr_t>(ws) & 255u) != 0)
+    return PQHSA_ERR_INVALID_ARG;
+  if (kv->stride_page % 8 || kv->stride_token % 8 || kv->stride_head % 8) return PQHSA_ERR_UNSUPPORTED;
+  if (pl.G > kMaxDenseWarps) return PQHSA_ERR_UNSUPPORTED;
+  if (ws_bytes < pqhsa_dense_workspace_bytes(params)) return PQHSA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  const size_t tick_bytes = align256d((size_t)pl.B * pl.Hkv * 4);
+  if (cudaMemsetAsync(w, 0, tick_bytes, st) != cudaSuccess) return PQHSA_ERR_CUDA;
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(w);
+  float* part = reinterpret_cast<float*>(w + tick_bytes);
+  const dim3 grid(dense_splits(pl), pl.Hkv, pl.B), block(32 * pl.G);
+  cudaError_t e;
+  if (pl.dtype == PQHSA_F16)
+    e = launch_pdl(dense_decode_kernel<__half, 4>, grid, block, 0, st, pl,
+                   static_cast<const __half*>(q), static_cast<const __half*>(kv->k_cache),
+                   static_cast<const __half*>(kv->v_cache), (long long)kv->stride_page,
+                   (long long)kv->stride_token, (long long)kv->stride_head, kv->block_table,
+                   seq_lens, part, tickets, static_cast<__half*>(out));
+  else
+    e = launch_pdl(dense_decode_kernel<__nv_bfloat16, 4>, grid, block, 0, st, pl,
+                   static_cast<const __nv_bfloat16*>(q),
+                   static_cast<const __nv_bfloat16*>(kv->k_cache),
+                   static_cast<const __nv_bfloat16*>(kv->v_cache), (long long)kv->stride_page,
+                   (long long)kv->stride_token, (long long)kv->stride_head, kv->block_table,
+                   seq_lens, part, tickets, static_cast<__nv_bfloat16*>(out));
+  return e == cudaSuccess ? PQHSA_OK : PQHSA_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -25,7 +25,8 @@ EXPORTS = [
     "pqhsa_build_lut", "pqhsa_scan", "pqhsa_select", "pqhsa_hybrid_attend", "pqhsa_decode",
     "pqhsa_decode_events", "pqhsa_decode_host", "pqhsa_last_device_status", "pqhsa_decode_buffer_offset",
     "pqhsa_decode_launch_count", "pqhsa_status_string", "pqhsa_select_static",
-    "pqhsa_select_static_bytes", "pqhsa_select_static_capacity",
+    "pqhsa_select_static_bytes", "pqhsa_select_static_capacity", "pqhsa_dense_decode",
+    "pqhsa_dense_workspace_bytes",
 ]
 
 
@@ -86,6 +87,8 @@ def lib() -> ctypes.CDLL:
             "pqhsa_select_static": (I, [P, V, V, V, V, V, V]),
             "pqhsa_select_static_bytes": (Z, [P]),
             "pqhsa_select_static_capacity": (Z, []),
+            "pqhsa_dense_decode": (I, [P, V, PK, V, V, V, Z, V]),
+            "pqhsa_dense_workspace_bytes": (Z, [P]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -228,6 +231,17 @@ def decode_events(params, q, index: Index, kv: PagedKV, seq_lens, out, ws, event
     _check("pqhsa_decode_events", lib().pqhsa_decode_events(
         ctypes.byref(params), _ptr(q), ctypes.byref(index), ctypes.byref(kv), _ptr(seq_lens),
         _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream), arr))
+
+
+def dense_workspace_bytes(params: Params) -> int:
+    return lib().pqhsa_dense_workspace_bytes(ctypes.byref(params))
+
+
+def dense_decode(params, q, kv: PagedKV, seq_lens, out, ws, stream=None) -> None:
+    """Dense decode attention over the whole paged cache (the sweep's comparator)."""
+    _check("pqhsa_dense_decode", lib().pqhsa_dense_decode(
+        ctypes.byref(params), _ptr(q), ctypes.byref(kv), _ptr(seq_lens), _ptr(out), _ptr(ws),
+        ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def decode_host(params, q_host, q_staging, index: Index, kv: PagedKV, seq_lens, out_staging,

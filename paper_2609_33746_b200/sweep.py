@@ -1,0 +1,67 @@
+"""Context-length sweep: PQ-HSA decode step against dense decode attention on the same paged
+cache (the crossover study of the paper's Sec. 4.4, on B200 and synthetic data).
+
+    python -m paper_2609_33746_b200.sweep [--contexts 16,32,64,128,256,512] [--batch 1] [--steps 50]
+
+Prints one JSON line per point: context, batch, us/step of pqhsa_decode and of
+pqhsa_dense_decode (CUDA events, L2 flushed between steps), their ratio, and bytes."""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import statistics
+
+import torch
+
+from . import pqhsa
+from .index_builder import build_index
+from .runner import DecodeOp
+from .workload import generate, named_config
+
+
+def time_call(fn, steps, flush):
+    for _ in range(3):
+        fn()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(steps)]
+    torch.cuda.synchronize()
+    for a, b in ev:
+        flush.zero_()
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return statistics.median(a.elapsed_time(b) for a, b in ev) * 1000.0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--contexts", default="16,32,64,128,256,512", help="context lengths in K tokens")
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--kmeans-iters", type=int, default=2)
+    args = ap.parse_args()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    for ctx in (int(x) for x in args.contexts.split(",")):
+        cfg = dataclasses.replace(named_config(f"c5_n{ctx}_b{args.batch}"),
+                                  kmeans_iters=args.kmeans_iters)
+        inp = generate(cfg, device="cuda")
+        idx = build_index(inp)
+        op = DecodeOp(inp, idx)
+        dws = torch.empty(pqhsa.dense_workspace_bytes(op.params), dtype=torch.uint8, device="cuda")
+        dout = torch.empty_like(op.q)
+        t_pq = time_call(op.decode, args.steps, flush)
+        t_dense = time_call(lambda: pqhsa.dense_decode(op.params, op.q, op.kv, op.seq_lens, dout,
+                                                       dws), args.steps, flush)
+        dense_bytes = cfg.batch * cfg.n_kv_heads * cfg.max_seq_len * 2 * cfg.head_dim * 2
+        print(json.dumps(dict(context=cfg.max_seq_len, batch=cfg.batch, n_list=cfg.n_list,
+                              budget_ppm=cfg.budget_ppm, pqhsa_us=round(t_pq, 1),
+                              dense_us=round(t_dense, 1), dense_over_pqhsa=round(t_dense / t_pq, 3),
+                              dense_gbs=round(dense_bytes / t_dense / 1e3, 1))), flush=True)
+        del op, inp, idx, dws
+        torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()

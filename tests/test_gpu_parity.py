@@ -319,3 +319,55 @@ def test_decode_host_entry_point_matches_device_entry_point():
     pqhsa.decode_host(op.params, q_host, q_stage, op.index, op.kv, op.seq_lens, out_stage,
                       out_host, op.ws)
     assert torch.allclose(out_host.float(), want.cpu().float(), atol=2e-3, rtol=2e-2)
+
+
+def test_decode_is_capturable_in_a_cuda_graph():
+    """The decode step makes no allocation and no synchronisation, so it can be captured once
+    and replayed (Sec. 3.3 replays the per-layer kernels as one CUDA graph)."""
+    inp, idx, arrays, ref, op = get_case("bf16_ragged_tail")
+    op.decode()
+    torch.cuda.synchronize()
+    want = op.out.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        op.decode()                                  # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        op.decode()
+    for _ in range(3):
+        op.out.fill_(5.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert op.device_status() == pqhsa.OK
+        assert torch.allclose(op.out.float(), want.float(), atol=2e-3, rtol=2e-2)
+
+
+@pytest.mark.parametrize("key", ["c1", "bf16_ragged_tail", "g8_two_head_groups", "ragged_batch_with_empty",
+                                 "interleaved_layout", "tiny"])
+def test_dense_comparator_is_textbook_attention(key):
+    """The dense decode kernel of the context sweep against softmax attention in float64."""
+    from scipy.special import softmax
+    inp, idx, arrays, ref, op = get_case(key)
+    cfg = inp.cfg
+    ws = torch.empty(pqhsa.dense_workspace_bytes(op.params), dtype=torch.uint8, device="cuda")
+    out = torch.full_like(op.q, 3.0)
+    pqhsa.dense_decode(op.params, op.q, op.kv, op.seq_lens, out, ws)
+    torch.cuda.synchronize()
+    got = out.cpu().double().numpy()
+    for b in range(cfg.batch):
+        n = int(arrays["seq_lens"][b])
+        for h in range(cfg.n_q_heads):
+            if n == 0:
+                assert np.all(got[b, h] == 0.0)
+                continue
+            g = h // cfg.group
+            pos = np.arange(n)
+            K = O.gather_rows(arrays["k_cache_flat"], arrays["block_table"][b], pos, g, 128,
+                              cfg.page_size, inp.stride_page, inp.stride_token, inp.stride_head)
+            V = O.gather_rows(arrays["v_cache_flat"], arrays["block_table"][b], pos, g, 128,
+                              cfg.page_size, inp.stride_page, inp.stride_token, inp.stride_head)
+            want = softmax(K @ arrays["q"][b, h] / math.sqrt(128.0)) @ V
+            assert np.all(np.abs(got[b, h] - want) <= out_tolerance(want, cfg.dtype))

@@ -131,7 +131,7 @@ void make_layout(const Plan& pl, WsLayout* L) {
   L->attend_zero_bytes = o - L->attend_tickets;
   L->zero_bytes = o - L->zero_begin;
   L->rowstate = take((size_t)pl.rows * 16);
-  L->cand = take((size_t)pl.rows * pl.cand_cap * 8);
+  L->cand = take((size_t)pl.rows * pl.cand_cap * 4);
   L->bg_max = take((size_t)pl.rows * 4);
   L->split_part = take((size_t)pl.rows * pl.splits * (2 + kHeadDim) * 4);
   L->stage_end = o;

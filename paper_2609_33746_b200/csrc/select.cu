@@ -130,43 +130,44 @@ __device__ __forceinline__ void load_chunk(const float* __restrict__ rs, int chu
 }
 
 // ------------------------------------------------------------------------- sample kernel
-// rank-th largest (0-based) of the CTA's 4096 sampled keys (8 per thread, in registers).
-__device__ uint32_t sample_order_stat(const uint32_t (&key)[kSamplePer], int rank,
-                                      uint32_t* s_hist, int* s_scan) {
+// 24-bit prefixes (key >> 8) of the rank_a-th and rank_b-th largest (0-based) of the CTA's 4096
+// sampled keys (8 per thread, in registers).  Two 12-bit digits; both ranks share each pass.
+__device__ void sample_prefixes(const uint32_t (&key)[kSamplePer], int rank_a, int rank_b,
+                                uint32_t* s_hist, uint32_t* s_hist_b, int* s_scan,
+                                uint32_t& pre_a, uint32_t& pre_b) {
   const int tid = threadIdx.x;
-  int need = rank + 1, d, above;
+  int d, above;
   for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
   __syncthreads();
 #pragma unroll
   for (int e = 0; e < kSamplePer; ++e) atomicAdd(&s_hist[key[e] >> 20], 1u);
   __syncthreads();
-  find_digit(s_hist, kHistBins, need, s_scan, d, above);
-  const uint32_t d1 = (uint32_t)d;
-  need -= above;
-  for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
+  find_digit(s_hist, kHistBins, rank_a + 1, s_scan, d, above);
+  const uint32_t a1 = (uint32_t)d;
+  const int need_a = rank_a + 1 - above;
+  find_digit(s_hist, kHistBins, rank_b + 1, s_scan, d, above);
+  const uint32_t b1 = (uint32_t)d;
+  const int need_b = rank_b + 1 - above;
+  for (int i = tid; i < kHistBins; i += kSelThreads) { s_hist[i] = 0u; s_hist_b[i] = 0u; }
   __syncthreads();
 #pragma unroll
-  for (int e = 0; e < kSamplePer; ++e)
-    if ((key[e] >> 20) == d1) atomicAdd(&s_hist[(key[e] >> 8) & 0xfffu], 1u);
+  for (int e = 0; e < kSamplePer; ++e) {
+    const uint32_t t = key[e] >> 20, lo12 = (key[e] >> 8) & 0xfffu;
+    if (t == a1) atomicAdd(&s_hist[lo12], 1u);
+    if (t == b1) atomicAdd(&s_hist_b[lo12], 1u);
+  }
   __syncthreads();
-  find_digit(s_hist, kHistBins, need, s_scan, d, above);
-  const uint32_t p2 = (d1 << 12) | (uint32_t)d;
-  need -= above;
-  for (int i = tid; i < 256; i += kSelThreads) s_hist[i] = 0u;
-  __syncthreads();
-#pragma unroll
-  for (int e = 0; e < kSamplePer; ++e)
-    if ((key[e] >> 8) == p2) atomicAdd(&s_hist[key[e] & 0xffu], 1u);
-  __syncthreads();
-  find_digit(s_hist, 256, need, s_scan, d, above);
-  return (p2 << 8) | (uint32_t)d;
+  find_digit(s_hist, kHistBins, need_a, s_scan, d, above);
+  pre_a = (a1 << 12) | (uint32_t)d;
+  find_digit(s_hist_b, kHistBins, need_b, s_scan, d, above);
+  pre_b = (b1 << 12) | (uint32_t)d;
 }
 
 __global__ void __launch_bounds__(kSelThreads)
 sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __restrict__ seq_lens,
                   int32_t* __restrict__ rowstate, int32_t* __restrict__ sel_count,
                   float* __restrict__ kth) {
-  __shared__ uint32_t s_hist[kHistBins];
+  __shared__ uint32_t s_hist[kHistBins], s_hist_b[kHistBins];
   __shared__ int s_scan[34];
   const int row = blockIdx.x, tid = threadIdx.x;
   const int b = row / pl.Hq;
@@ -203,8 +204,15 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
     const float r = p * kSample;
     const int mgn = (int)ceilf(kBracketSigmas * sqrtf(kSample * p * (1.f - p))) + 2;
     const int r_hi = (int)floorf(r) - mgn, r_lo = (int)ceilf(r) + mgn;
-    if (r_hi >= 0) hi = key_score(sample_order_stat(key, r_hi, s_hist, s_scan));
-    if (r_lo < kSample) lo = key_score(sample_order_stat(key, r_lo, s_hist, s_scan));
+    // the bracket only has to contain the two order statistics: take the edges of their
+    // 24-bit key prefixes (256 ulps wide), which saves the third radix digit
+    uint32_t pre_hi, pre_lo;
+    sample_prefixes(key, max(r_hi, 0), min(r_lo, kSample - 1), s_hist, s_hist_b, s_scan, pre_hi,
+                    pre_lo);
+    if (r_hi >= 0) hi = key_score((pre_hi << 8) | 0xffu);
+    if (r_lo < kSample) lo = key_score(pre_lo << 8);
+    if (hi != hi) hi = CUDART_INF_F;                 // prefix that runs into the NaN patterns
+    if (lo != lo) lo = -CUDART_INF_F;
   }
   if (tid == 0) {
     rowstate[row * 4 + 0] = __float_as_int(lo);
@@ -218,10 +226,11 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
 enum Source { kFromStash = 0, kFromList = 1, kFromRow = 2 };
 
 // Calls f(valid, key, position) for every item of the source: the candidates staged in
-// shared memory, the candidate list in global memory, or the whole score row.  Uniform trip
+// shared memory as (key, position), the candidate list in global memory (positions; the key
+// comes from the score row), or the whole score row.  Uniform trip
 // count: f may use warp votes.
 template <class F>
-__device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, const uint2* cand,
+__device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, const int32_t* cand,
                                               int n_items, const float* rs, F f) {
   const int tid = threadIdx.x;
   constexpr int U = 4;
@@ -234,17 +243,19 @@ __device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, con
     }
   } else if (src == kFromList) {
     for (int base = 0; base < n_items; base += kSelThreads * U) {
-      uint2 c[U];
+      int pos[U];
+      float sc[U];
       bool v[U];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int i = base + u * kSelThreads + tid;
         v[u] = i < n_items;
-        c[u] = make_uint2(0u, 0u);
-        if (v[u]) c[u] = __ldcg(cand + i);
+        pos[u] = v[u] ? __ldcg(cand + i) : 0;
       }
 #pragma unroll
-      for (int u = 0; u < U; ++u) f(v[u], c[u].x, (int)c[u].y);
+      for (int u = 0; u < U; ++u) sc[u] = v[u] ? __ldcg(rs + pos[u]) : 0.f;
+#pragma unroll
+      for (int u = 0; u < U; ++u) f(v[u], score_key(sc[u]), pos[u]);
     }
   } else {
     for (int base = 0; base < n_items; base += kSelThreads * U) {
@@ -265,7 +276,7 @@ __device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, con
 // Exact selection of the `r` largest of the source's items (ties: lowest position), appended
 // to out[base_out ...].  Radix digits 12 / 12 / 8.  Returns the key of the r-th largest.
 // Runs in one CTA; 1 <= r <= n_items.
-__device__ uint32_t resolve_top_r(int src, const uint2* s_stash, const uint2* cand, int n_items,
+__device__ uint32_t resolve_top_r(int src, const uint2* s_stash, const int32_t* cand, int n_items,
                                   const float* rs, int n, int r, int32_t* out, uint32_t base_out,
                                   int k_max, uint32_t* s_hist, int* s_scan, uint32_t* s_emit) {
   const int tid = threadIdx.x;
@@ -333,11 +344,15 @@ __device__ uint32_t resolve_top_r(int src, const uint2* s_stash, const uint2* ca
 
 __global__ void __launch_bounds__(kSelThreads, 3)
 sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restrict__ counters,
-                  const int32_t* __restrict__ rowstate, uint2* __restrict__ cand,
+                  const int32_t* __restrict__ rowstate, int32_t* __restrict__ cand,
                   int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_count,
                   float* __restrict__ kth, int* __restrict__ status) {
-  __shared__ uint32_t s_hist[kHistBins];
-  __shared__ uint2 s_stash[kStashCap];
+  // main pass: a 512-entry hit buffer per warp; last CTA: histogram + candidate stash.
+  // The two uses never overlap in time, so they share the same shared memory.
+  __shared__ __align__(16) unsigned char s_raw[kHistBins * 4 + kStashCap * 8];
+  uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_raw);
+  uint2* s_stash = reinterpret_cast<uint2*>(s_raw + kHistBins * 4);
+  uint32_t* s_hits = reinterpret_cast<uint32_t*>(s_raw);          // [16 warps][512]
   __shared__ int s_scan[34];
   __shared__ int s_last;
   __shared__ uint32_t s_emit;
@@ -351,68 +366,78 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
   if (k == 0) return;
   const float* rs = scores + (size_t)row * pl.N_max;
   int32_t* out = sel_idx + (size_t)row * pl.k_max;
-  uint2* rc = cand + (size_t)row * pl.cand_cap;
+  int32_t* rc = cand + (size_t)row * pl.cand_cap;
   uint32_t* n_out = &counters[row * 4 + 2];
   uint32_t* n_cand = &counters[row * 4 + 3];
 
-  // Main pass.  Warps work independently: classify 16 scores per lane, take output slots
-  // with one atomic per warp and list, write.  No block-wide barrier inside the loop.
+  // Main pass.  Warps work independently: a lane marks which of its 16 scores reach the
+  // bracket, the warp packs the positions of the hits (bit 31 = certain winner) into its
+  // shared-memory buffer, and flushes them with one atomic per destination list.
   const int n_chunks = (n + kSelChunk - 1) / kSelChunk;
   const bool no_winners = !(hi_f < CUDART_INF_F);   // bracket open at the top: candidates only
+  uint32_t* my_hits = s_hits + warp * (kSelChunk / 16);
   for (int ch = chunk; ch < n_chunks; ch += gridDim.x) {
     float v[kElems];
     int pos0[4];
     load_chunk(rs, ch, n, v, pos0);
     const bool full = (ch + 1) * kSelChunk <= n;
-    uint32_t win_mask = 0, cand_mask = 0;
+    uint32_t hit = 0, win = 0;
     if (full && no_winners) {
 #pragma unroll
-      for (int e = 0; e < kElems; ++e) cand_mask |= (v[e] >= lo_f ? 1u : 0u) << e;
+      for (int e = 0; e < kElems; ++e) hit |= (v[e] >= lo_f ? 1u : 0u) << e;
     } else {
 #pragma unroll
       for (int e = 0; e < kElems; ++e) {
         const bool valid = full || pos0[e >> 2] + (e & 3) < n;
-        const bool win = v[e] > hi_f;
-        win_mask |= (valid && win ? 1u : 0u) << e;
-        cand_mask |= (valid && !win && v[e] >= lo_f ? 1u : 0u) << e;
+        hit |= (valid && v[e] >= lo_f ? 1u : 0u) << e;
+        win |= (valid && v[e] > hi_f ? 1u : 0u) << e;
       }
     }
-    // inclusive scan of (winners << 16 | candidates) over the warp; lane 31 takes the slots
-    const uint32_t mine = ((uint32_t)__popc(win_mask) << 16) | (uint32_t)__popc(cand_mask);
-    uint32_t inc = mine;
+    // exclusive scan of the per-lane hit counts over the warp
+    const int mine = __popc(hit);
+    int inc = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t u = __shfl_up_sync(0xffffffffu, inc, o);
+      const int u = __shfl_up_sync(0xffffffffu, inc, o);
       if (lane >= o) inc += u;
     }
-    uint32_t base_w = 0, base_c = 0;
-    if (lane == 31) {
-      const uint32_t tw = inc >> 16, tc = inc & 0xffffu;
-      if (tw) base_w = atomicAdd(n_out, tw);
-      if (tc) base_c = atomicAdd(n_cand, tc);
+    const int total = __shfl_sync(0xffffffffu, inc, 31);
+    if (total == 0) continue;                        // warp-uniform
+    int slot = inc - mine;
+    const int pos_base = ch * kSelChunk + tid * 4;   // position of element e: + (e>>2)*2048 + (e&3)
+    while (hit) {
+      const int e = __ffs(hit) - 1;
+      hit &= hit - 1;
+      my_hits[slot++] = (uint32_t)(pos_base + (e >> 2) * (kSelThreads * 4) + (e & 3)) |
+                        (((win >> e) & 1u) << 31);
     }
-    base_w = __shfl_sync(0xffffffffu, base_w, 31);
-    base_c = __shfl_sync(0xffffffffu, base_c, 31);
-    uint32_t pw = base_w + ((inc - mine) >> 16), pc = base_c + ((inc - mine) & 0xffffu);
-    if (win_mask) {
-#pragma unroll
-      for (int e = 0; e < kElems; ++e) {
-        if (win_mask & (1u << e)) {
-          if (pw < (uint32_t)pl.k_max) out[pw] = pos0[e >> 2] + (e & 3);
-          ++pw;
-        }
+    __syncwarp();
+    for (int i0 = 0; i0 < total; i0 += 32) {
+      const int i = i0 + lane;
+      const bool v_ok = i < total;
+      const uint32_t ent = v_ok ? my_hits[i] : 0u;
+      const bool is_win = v_ok && (ent >> 31);
+      const bool is_cnd = v_ok && !(ent >> 31);
+      const unsigned mw = __ballot_sync(0xffffffffu, is_win);
+      const unsigned mc = __ballot_sync(0xffffffffu, is_cnd);
+      uint32_t bw = 0, bc = 0;
+      if (lane == 0) {
+        if (mw) bw = atomicAdd(n_out, (uint32_t)__popc(mw));
+        if (mc) bc = atomicAdd(n_cand, (uint32_t)__popc(mc));
+      }
+      bw = __shfl_sync(0xffffffffu, bw, 0);
+      bc = __shfl_sync(0xffffffffu, bc, 0);
+      const unsigned lt = (1u << lane) - 1u;
+      if (is_win) {
+        const uint32_t p = bw + __popc(mw & lt);
+        if (p < (uint32_t)pl.k_max) out[p] = (int)(ent & 0x7fffffffu);
+      }
+      if (is_cnd) {
+        const uint32_t p = bc + __popc(mc & lt);
+        if (p < (uint32_t)pl.cand_cap) rc[p] = (int)ent;
       }
     }
-    if (cand_mask) {
-#pragma unroll
-      for (int e = 0; e < kElems; ++e) {
-        if (cand_mask & (1u << e)) {
-          if (pc < (uint32_t)pl.cand_cap)
-            rc[pc] = make_uint2(score_key(v[e]), (uint32_t)(pos0[e >> 2] + (e & 3)));
-          ++pc;
-        }
-      }
-    }
+    __syncwarp();
   }
   __threadfence();
   __syncthreads();
@@ -444,7 +469,20 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
     } else {
       int src = kFromList;
       if (C <= kStashCap) {
-        for (int i = tid; i < C; i += kSelThreads) s_stash[i] = __ldcg(rc + i);
+        constexpr int kPer = kStashCap / kSelThreads;          // 6: all loads issued together
+        int pos[kPer];
+        float sc[kPer];
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+          const int i = u * kSelThreads + tid;
+          pos[u] = i < C ? __ldcg(rc + i) : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) sc[u] = pos[u] >= 0 ? __ldcg(rs + pos[u]) : 0.f;
+#pragma unroll
+        for (int u = 0; u < kPer; ++u)
+          if (pos[u] >= 0)
+            s_stash[u * kSelThreads + tid] = make_uint2(score_key(sc[u]), (uint32_t)pos[u]);
         __syncthreads();
         src = kFromStash;
       }
@@ -472,7 +510,7 @@ cudaError_t launch_select(const Plan& pl, const WsLayout& L, char* ws, const flo
                           float* kth, cudaStream_t st) {
   uint32_t* counters = reinterpret_cast<uint32_t*>(ws + L.counters);
   int32_t* rowstate = reinterpret_cast<int32_t*>(ws + L.rowstate);
-  uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
+  int32_t* cand = reinterpret_cast<int32_t*>(ws + L.cand);
   int* status = reinterpret_cast<int*>(ws + L.status);
   cudaError_t e = launch_pdl(sel_sample_kernel, dim3(pl.rows), dim3(kSelThreads), 0, st, pl, scores,
                              seq_lens, rowstate, sel_count, kth);

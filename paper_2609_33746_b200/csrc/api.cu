@@ -3,6 +3,7 @@
 // except pqhsa_last_device_status and pqhsa_decode_host, which say so.
 #include <mutex>
 
+#include <cstdlib>
 #include "common.cuh"
 
 namespace pqhsa {
@@ -91,18 +92,32 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (o.hist_chunks < 1) o.hist_chunks = 1;
   o.cand_cap = o.N_max / 4 > kSelChunk ? o.N_max / 4 : kSelChunk;
   if (o.cand_cap > o.N_max) o.cand_cap = o.N_max;
-  // split-K CTAs per row: about 256 selected tokens each, but enough CTAs to fill the GPU
-  // when there are few rows, as long as every CTA keeps at least 32 units of work
-  o.splits = ceil_div(o.k_max, 256);
-  int fill = (4 * o.num_sms) / o.rows;     // one wave of resident CTAs (4 per SM)
-  const int max_fill = (o.k_max + o.n_list / 4) / 32 > 0 ? (o.k_max + o.n_list / 4) / 32 : 1;
+  // attend kernel, background CTAs per (sequence, KV head, head group): about two per SM in
+  // total, at least 32 lists each
+  o.bg_splits = ceil_div(2LL * o.num_sms, (long long)o.B * o.upb);
+  if (o.bg_splits > o.n_list / 32) o.bg_splits = o.n_list / 32;
+  if (o.bg_splits > 16) o.bg_splits = 16;
+  if (o.bg_splits < 1) o.bg_splits = 1;
+  // attend kernel, split-K CTAs per row: about 512 selected tokens each, but enough CTAs to
+  // fill the GPU when there are few rows (one wave of 4 resident CTAs per SM, background
+  // CTAs included), as long as every CTA keeps at least 32 tokens
+  o.splits = ceil_div(o.k_max, 512);
+  int fill = (4 * o.num_sms - o.B * o.upb * o.bg_splits) / o.rows;
+  const int max_fill = o.k_max / 32 > 0 ? o.k_max / 32 : 1;
   if (fill > max_fill) fill = max_fill;
   if (o.splits < fill) o.splits = fill;
   if (o.splits > 64) o.splits = 64;
   if (o.splits < 1) o.splits = 1;
+  // background preparation: CTAs per row
   o.bg_ctas = ceil_div(2LL * o.num_sms, o.rows);
   if (o.bg_ctas > 8) o.bg_ctas = 8;
   if (o.bg_ctas < 1) o.bg_ctas = 1;
+#ifdef PQHSA_TUNE
+  if (const char* e = getenv("PQHSA_HIST_CHUNKS")) o.hist_chunks = atoi(e);
+  if (const char* e = getenv("PQHSA_SPLITS")) o.splits = atoi(e);
+  if (const char* e = getenv("PQHSA_BG_CTAS")) o.bg_ctas = atoi(e);
+  if (const char* e = getenv("PQHSA_BG_SPLITS")) o.bg_splits = atoi(e);
+#endif
   return PQHSA_OK;
 }
 
@@ -133,7 +148,7 @@ void make_layout(const Plan& pl, WsLayout* L) {
   L->rowstate = take((size_t)pl.rows * 16);
   L->cand = take((size_t)pl.rows * pl.cand_cap * 4);
   L->bg_max = take((size_t)pl.rows * 4);
-  L->split_part = take((size_t)pl.rows * pl.splits * (2 + kHeadDim) * 4);
+  L->split_part = take((size_t)pl.rows * (pl.splits + pl.bg_splits) * (4 + kHeadDim) * 4);
   L->stage_end = o;
   L->lut = take(buffer_elems(pl, PQHSA_BUF_LUT) * 4);
   L->coarse = take(buffer_elems(pl, PQHSA_BUF_COARSE) * 4);
@@ -232,7 +247,7 @@ int pqhsa_decode_launch_count(const pqhsa_params* params) {
   Plan pl;
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
-  return 6;   // LUT build, scan, select sample, select filter, background prep, attend
+  return 6;   // LUT build, scan, select sample, select filter, attend exact, attend background
 }
 
 int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index* index,

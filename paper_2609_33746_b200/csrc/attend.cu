@@ -18,7 +18,6 @@ namespace pqhsa {
 namespace {
 
 constexpr int kBgThreads = 256;
-constexpr int kPartStride = 2 + kHeadDim;     // m, Z, N[128]
 constexpr int kMaxSeg = 160;                  // >= n_part for any plan (148 SMs / 1 unit + 2)
 
 // grid (bg_ctas, rows).  CTA c merges a slice of the lists and subtracts a slice of the
@@ -112,6 +111,17 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   if (c == 0 && tid == 0) bg_max[row] = m;
 }
 
+// One grid, two kinds of CTA.
+//   CTAs [0, rows * S): split s of score row r gathers its share of the selected K/V rows
+//     (8 lanes per 256-byte row, 16 rows in flight per warp, positions and page ids fetched
+//     one 32-token window ahead) and keeps an online softmax in base 2.  These CTAs read
+//     only what the top-k wrote, so they do not wait for the background preparation, which
+//     runs while they gather.
+//   CTAs [rows * S, rows * S + units * BS): slice c of the lists of one (sequence, KV head,
+//     head group): Z += M_j, N += M_j * vbar_j for the up to 4 heads of the group from one
+//     read of the vbar rows.  These wait for the background preparation.
+// Every CTA leaves one partial per row it worked for and takes a ticket of that row; the
+// CTA that draws the last ticket merges the row (nobody waits).
 template <typename T, int U>
 __global__ void __launch_bounds__(kAttendThreads, 4)
 attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
@@ -122,21 +132,91 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
               float* __restrict__ split_part, uint32_t* __restrict__ tickets,
               T* __restrict__ out, float* __restrict__ lse) {
   constexpr int kWarps = kAttendThreads / 32;
-  __shared__ float s_m[2 * kWarps], s_Z[2 * kWarps];
-  __shared__ __align__(16) float s_N[2 * kWarps][kHeadDim];
-  __shared__ int s_last;
+  __shared__ float s_m[kWarps], s_Z[4 * kWarps];
+  __shared__ __align__(16) float s_N[4 * kWarps][kHeadDim];
+  __shared__ int s_last[4];
+  __shared__ float s_aux[kMaxParts + 8];
 
-  const int split = blockIdx.x, S = gridDim.x, row = blockIdx.y;
+  const int S = pl.splits, BS = pl.bg_splits, n_part = S + BS;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = row / pl.Hq, h = row % pl.Hq, kv = h / pl.G;
-  const size_t ukv = (size_t)b * pl.Hkv + kv;
   const int n_list = pl.n_list;
-  pdl_wait();
+
+  if ((int)blockIdx.x >= pl.rows * S) {
+    // ================= background CTA =================
+    const int id = (int)blockIdx.x - pl.rows * S;
+    const int unit = id / BS, c = id % BS;                  // unit = (b, kv, head group)
+    const int hg = unit % pl.n_hg, kv = (unit / pl.n_hg) % pl.Hkv, b = unit / (pl.n_hg * pl.Hkv);
+    const int h0 = kv * pl.G + hg * pl.Gc;                  // first head of the group
+    const int n_heads = min(pl.Gc, pl.G - hg * pl.Gc);
+    const int row0 = b * pl.Hq + h0;
+    pdl_wait();
+    pdl_launch_dependents();
+    const int jl = (int)((long long)c * n_list / BS), jh = (int)((long long)(c + 1) * n_list / BS);
+    const int per = (jh - jl + kWarps - 1) / kWarps;
+    const int a = min(jh, jl + warp * per), e = min(jh, a + per);
+    const float4* vm = reinterpret_cast<const float4*>(
+        vmeans + ((size_t)b * pl.Hkv + kv) * n_list * kHeadDim);
+    // lane (g, i) = (lane >> 3, lane & 7) fetches the mass of head g for list j0 + i
+    const int mg = lane >> 3, mi = lane & 7;
+    const float* mass = bg_mass + (size_t)(row0 + (mg < n_heads ? mg : 0)) * n_list;
+    float4 acc[4];
+    float z = 0.f;                                          // lane (g, *) sums head g's masses
+#pragma unroll
+    for (int g = 0; g < 4; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j0 = a; j0 < e; j0 += 8) {
+      const float mine = (mg < n_heads && j0 + mi < e) ? fmaxf(mass[j0 + mi], 0.f) : 0.f;
+      const unsigned nz = __ballot_sync(0xffffffffu, mine > 0.f);
+      const unsigned live = (nz | (nz >> 8) | (nz >> 16) | (nz >> 24)) & 0xffu;   // any head
+      float4 v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if ((live >> i) & 1u) v[i] = __ldg(vm + (size_t)(j0 + i) * (kHeadDim / 4) + lane);
+      }
+      z += mine;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const float mj = __shfl_sync(0xffffffffu, mine, 8 * g + i);
+          acc[g].x = fmaf(mj, v[i].x, acc[g].x); acc[g].y = fmaf(mj, v[i].y, acc[g].y);
+          acc[g].z = fmaf(mj, v[i].z, acc[g].z); acc[g].w = fmaf(mj, v[i].w, acc[g].w);
+        }
+      }
+    }
+    z += __shfl_xor_sync(0xffffffffu, z, 1);
+    z += __shfl_xor_sync(0xffffffffu, z, 2);
+    z += __shfl_xor_sync(0xffffffffu, z, 4);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) *reinterpret_cast<float4*>(&s_N[4 * warp + g][4 * lane]) = acc[g];
+    if (mi == 0) s_Z[4 * warp + mg] = z;
+    __syncthreads();
+    for (int g = 0; g < n_heads; ++g) {
+      float Z_c = 0.f, N_c = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) { Z_c += s_Z[4 * w + g]; N_c += s_N[4 * w + g][tid]; }
+      float* part = split_part + ((size_t)(row0 + g) * n_part + S + c) * kPartStride;
+      part[4 + tid] = N_c;
+      if (tid == 0) { part[0] = bg_max[row0 + g] * kLog2e; part[1] = Z_c; }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid < n_heads) s_last[tid] = (atomicAdd(&tickets[row0 + tid], 1u) == (uint32_t)(n_part - 1));
+    __syncthreads();
+    for (int g = 0; g < n_heads; ++g) {
+      if (!s_last[g]) continue;
+      __threadfence();
+      merge_row(split_part + (size_t)(row0 + g) * n_part * kPartStride, n_part, row0 + g, tid,
+                s_N, s_aux, out, lse);
+    }
+    return;
+  }
+
+  // ================= exact (selected-token) CTA =================
+  const int row = (int)blockIdx.x / S, split = (int)blockIdx.x % S;
+  const int b = row / pl.Hq, h = row % pl.Hq, kv = h / pl.G;
   pdl_launch_dependents();
   const int cnt = sel_count[row];
-
-  // ---- this warp's slice of the selected tokens: resolve cache offsets first (two
-  //      dependent loads: position, then page id), so they overlap the background part
   const int tl = (int)((long long)split * cnt / S);
   const int th = (int)((long long)(split + 1) * cnt / S);
   const int per_warp = (th - tl + kWarps - 1) / kWarps;
@@ -145,50 +225,6 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   const int32_t* bt = block_table + (size_t)b * pl.max_pages;
   int my_pos = (wl + lane < wh) ? sel[wl + lane] : -1;
 
-  const float m_bg = bg_max[row] * kLog2e;    // reference of the background masses (log2 units)
-
-  // ---- background slice: Z += M_j, N += M_j * vbar_j  (all relative to m_bg)
-  {
-    const int jl = (int)((long long)split * n_list / S);
-    const int jh = (int)((long long)(split + 1) * n_list / S);
-    const int per = (jh - jl + kWarps - 1) / kWarps;
-    const int a = min(jh, jl + warp * per), e = min(jh, a + per);
-    const float* mass = bg_mass + (size_t)row * n_list;
-    const float4* vm = reinterpret_cast<const float4*>(vmeans + ukv * n_list * kHeadDim);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float z = 0.f;
-    for (int j0 = a; j0 < e; j0 += 32) {
-      const float mine = (j0 + lane < e) ? fmaxf(mass[j0 + lane], 0.f) : 0.f;
-      unsigned live = __ballot_sync(0xffffffffu, mine > 0.f);
-      while (live) {
-        int jj[4];
-        float mj[4];
-        float4 v[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          jj[u] = live ? __ffs(live) - 1 : -1;
-          if (live) live &= live - 1;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          mj[u] = __shfl_sync(0xffffffffu, mine, jj[u] < 0 ? 0 : jj[u]);
-          v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (jj[u] >= 0) v[u] = __ldg(vm + (size_t)(j0 + jj[u]) * (kHeadDim / 4) + lane);
-          else mj[u] = 0.f;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          acc.x = fmaf(mj[u], v[u].x, acc.x); acc.y = fmaf(mj[u], v[u].y, acc.y);
-          acc.z = fmaf(mj[u], v[u].z, acc.z); acc.w = fmaf(mj[u], v[u].w, acc.w);
-          z += mj[u];
-        }
-      }
-    }
-    *reinterpret_cast<float4*>(&s_N[kWarps + warp][4 * lane]) = acc;
-    if (lane == 0) { s_m[kWarps + warp] = m_bg; s_Z[kWarps + warp] = z; }
-  }
-
-  // ---- exact slice
   const int gi = lane >> 3, gl = lane & 7;      // lane group (4 per warp) and lane in group
   float qf[16];
   {
@@ -201,13 +237,13 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
     }
   }
   GroupState st;
-  st.m = m_bg;
+  st.m = -CUDART_INF_F;
   st.Z = 0.f;
 #pragma unroll
   for (int t = 0; t < 16; ++t) st.acc[t] = 0.f;
 
-  // page id of this lane's first token (second dependent load); later batches prefetch
-  // position and page one batch ahead, while the current batch's rows are in flight
+  // page id of this lane's first token (second dependent load); later windows prefetch
+  // position and page one window ahead, while the current window's rows are in flight
   int my_page = my_pos >= 0 ? __ldg(bt + my_pos / pl.page_size) : 0;
   for (int base = wl; base < wh; base += 32) {
     long long off = 0;
@@ -250,7 +286,7 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
         s += __shfl_xor_sync(0xffffffffu, s, 4);
         if (ok[u]) {                                  // uniform within the lane group
           if (s > st.m) {
-            const float a = fast_exp2(st.m - s);
+            const float a = st.Z > 0.f ? fast_exp2(st.m - s) : 0.f;
             st.Z *= a;
 #pragma unroll
             for (int t = 0; t < 16; ++t) st.acc[t] *= a;
@@ -299,49 +335,24 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   // ---- CTA partial: thread d owns output dim d
   float m_c = -CUDART_INF_F;
 #pragma unroll
-  for (int w = 0; w < 2 * kWarps; ++w) if (s_Z[w] > 0.f) m_c = fmaxf(m_c, s_m[w]);
+  for (int w = 0; w < kWarps; ++w) if (s_Z[w] > 0.f) m_c = fmaxf(m_c, s_m[w]);
   float Z_c = 0.f, N_c = 0.f;
 #pragma unroll
-  for (int w = 0; w < 2 * kWarps; ++w) {
+  for (int w = 0; w < kWarps; ++w) {
     const float a = safe_scale(s_m[w], m_c, s_Z[w]);
     Z_c = fmaf(s_Z[w], a, Z_c);
     N_c = fmaf(s_N[w][tid], a, N_c);
   }
-  float* part = split_part + ((size_t)row * S + split) * kPartStride;
-  part[2 + tid] = N_c;
+  float* part = split_part + ((size_t)row * n_part + split) * kPartStride;
+  part[4 + tid] = N_c;
   if (tid == 0) { part[0] = m_c; part[1] = Z_c; }
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&tickets[row], 1u) == (uint32_t)(S - 1));
+  if (tid == 0) s_last[0] = (atomicAdd(&tickets[row], 1u) == (uint32_t)(n_part - 1));
   __syncthreads();
-  if (!s_last) return;
+  if (!s_last[0]) return;
   __threadfence();
-
-  // ---- last CTA of the row: merge the S partials and normalise (Eq. 5)
-  const float* pr = split_part + (size_t)row * S * kPartStride;
-  float m_r = -CUDART_INF_F;
-  for (int s = 0; s < S; ++s)
-    if (__ldcg(pr + s * kPartStride + 1) > 0.f) m_r = fmaxf(m_r, __ldcg(pr + s * kPartStride));
-  float Z_r = 0.f, N_r = 0.f;
-  for (int s0 = 0; s0 < S; s0 += 4) {
-    float Zs[4], ms[4], Ns[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int s = s0 + u;
-      Zs[u] = s < S ? __ldcg(pr + s * kPartStride + 1) : 0.f;
-      ms[u] = s < S ? __ldcg(pr + s * kPartStride) : 0.f;
-      Ns[u] = s < S ? __ldcg(pr + s * kPartStride + 2 + tid) : 0.f;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const float a = safe_scale(ms[u], m_r, Zs[u]);
-      Z_r = fmaf(Zs[u], a, Z_r);
-      N_r = fmaf(Ns[u], a, N_r);
-    }
-  }
-  out[(size_t)row * kHeadDim + tid] = Unpack<T>::pack(Z_r > 0.f ? N_r / Z_r : 0.f);
-  if (lse != nullptr && tid == 0)
-    lse[row] = Z_r > 0.f ? (m_r + log2f(Z_r)) / kLog2e : -CUDART_INF_F;
+  merge_row(split_part + (size_t)row * n_part * kPartStride, n_part, row, tid, s_N, s_aux, out, lse);
 }
 
 }  // namespace
@@ -359,7 +370,7 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
                              scores, list_partials, sel_idx, sel_count, ix.list_ids, seq_lens,
                              bg_mass, bg_max);
   if (e != cudaSuccess) return e;
-  dim3 grid(pl.splits, pl.rows);
+  dim3 grid(pl.rows * pl.splits + pl.B * pl.Hkv * pl.n_hg * pl.bg_splits);
   if (pl.dtype == PQHSA_F16)
     return launch_pdl(attend_kernel<__half, 4>, grid, dim3(kAttendThreads), 0, st, pl,
                       static_cast<const __half*>(q), static_cast<const __half*>(kv.k_cache),

@@ -44,5 +44,68 @@ __device__ __forceinline__ float safe_scale(float m_from, float m_to, float Z) {
   return Z > 0.f ? fast_exp2(m_from - m_to) : 0.f;
 }
 
+// Split-K partial of one score row: m (log2 units), Z, two pad words, N[128] (16-byte aligned).
+constexpr int kPartStride = 4 + kHeadDim;
+constexpr int kMaxParts = 128;       // partials per row a 128-thread merge can take
+
+// Merges the n_part <= 128 partials of one row and writes y = N / Z (Eq. 5) and, if asked,
+// the log-sum-exp.  Called by all 128 threads of the CTA that finished last for the row,
+// after a fence.  Every load of a phase is independent (one L2 round trip per phase): thread
+// t fetches (m, Z) of partial t; then warp w sums N of partials w, w + 4, ..., a lane owning
+// 4 dims; shared memory joins the four warps.  s_red: 4 x 128 floats, s_aux: 128 + 8 floats.
+template <typename T>
+__device__ __forceinline__ void merge_row(const float* __restrict__ pr, int n_part, int row,
+                                          int tid, float (*s_red)[kHeadDim], float* s_aux,
+                                          T* __restrict__ out, float* __restrict__ lse) {
+  const int lane = tid & 31, warp = tid >> 5;
+  float m_t = -CUDART_INF_F, Z_t = 0.f;
+  if (tid < n_part) {
+    const float2 mz = __ldcg(reinterpret_cast<const float2*>(pr + (size_t)tid * kPartStride));
+    m_t = mz.x;
+    Z_t = mz.y;
+  }
+  float m_w = Z_t > 0.f ? m_t : -CUDART_INF_F;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(0xffffffffu, m_w, o));
+  __syncthreads();                      // callers may still be reading s_red / s_aux
+  if (lane == 0) s_aux[kMaxParts + warp] = m_w;
+  __syncthreads();
+  const float m_r = fmaxf(fmaxf(s_aux[kMaxParts], s_aux[kMaxParts + 1]),
+                          fmaxf(s_aux[kMaxParts + 2], s_aux[kMaxParts + 3]));
+  const float a_t = safe_scale(m_t, m_r, Z_t);
+  s_aux[tid] = a_t;
+  float Z_w = Z_t * a_t;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) Z_w += __shfl_xor_sync(0xffffffffu, Z_w, o);
+  if (lane == 0) s_aux[kMaxParts + 4 + warp] = Z_w;
+  __syncthreads();
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = warp; s0 < n_part; s0 += 32) {
+    float4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int s = s0 + 4 * u;
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (s < n_part)
+        v[u] = __ldcg(reinterpret_cast<const float4*>(pr + (size_t)s * kPartStride + 4) + lane);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int s = s0 + 4 * u;
+      const float a = s < n_part ? s_aux[s] : 0.f;
+      acc.x = fmaf(v[u].x, a, acc.x); acc.y = fmaf(v[u].y, a, acc.y);
+      acc.z = fmaf(v[u].z, a, acc.z); acc.w = fmaf(v[u].w, a, acc.w);
+    }
+  }
+  *reinterpret_cast<float4*>(&s_red[warp][4 * lane]) = acc;
+  __syncthreads();
+  const float Z_r = s_aux[kMaxParts + 4] + s_aux[kMaxParts + 5] + s_aux[kMaxParts + 6] +
+                    s_aux[kMaxParts + 7];
+  const float N_r = s_red[0][tid] + s_red[1][tid] + s_red[2][tid] + s_red[3][tid];
+  out[(size_t)row * kHeadDim + tid] = Unpack<T>::pack(Z_r > 0.f ? N_r / Z_r : 0.f);
+  if (lse != nullptr && tid == 0)
+    lse[row] = Z_r > 0.f ? (m_r + log2f(Z_r)) / kLog2e : -CUDART_INF_F;
+}
+
 }  // namespace
 }  // namespace pqhsa

@@ -41,7 +41,8 @@ struct Plan {
   int rows;                          // B * Hq score rows
   int hist_chunks;                   // CTAs per row in the select kernels
   int cand_cap;                      // candidate slots per row
-  int splits;                        // split-K CTAs per row in the attend kernel
+  int splits;                        // exact (split-K) CTAs per row in the attend kernel
+  int bg_splits;                     // background CTAs per (sequence, KV head, head group) there
   int bg_ctas;                       // CTAs per row in the background preparation
   int coarse_in_smem;                // scan keeps the coarse table in shared memory
   int scan_stages;                   // cp.async stages per warp in the scan's code ring (3 or 2)
@@ -59,7 +60,7 @@ struct WsLayout {
   size_t cand;                       // int32  [rows][cand_cap]: candidate positions
   size_t bg_mass;                    // float  [rows][n_list]: M_j relative to bg_max (accumulated)
   size_t bg_max;                     // float  [rows]
-  size_t split_part;                 // float  [rows][splits][2 + 128]: m, Z, N[128]
+  size_t split_part;                 // float  [rows][splits + bg_splits][4 + 128]: m, Z, pad, N[128]
   size_t stage_end;                  // end of what a single stage call needs
   // intermediates of the fused entry point
   size_t lut, coarse, scores, list_partials, sel_idx, sel_count, kth;

@@ -14,7 +14,7 @@ namespace pqhsa {
 
 namespace {
 
-constexpr int kDensePart = 2 + kHeadDim;
+constexpr int kDensePart = kPartStride;
 constexpr int kMaxDenseWarps = 16;
 
 template <typename T, int U>
@@ -130,8 +130,8 @@ dense_decode_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc,
   if (gi == 0) {
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
-      pr[2 + 8 * gl + t] = st.acc[t];
-      pr[2 + 64 + 8 * gl + t] = st.acc[8 + t];
+      pr[4 + 8 * gl + t] = st.acc[t];
+      pr[4 + 64 + 8 * gl + t] = st.acc[8 + t];
     }
     if (gl == 0) { pr[0] = st.m; pr[1] = st.Z; }
   }
@@ -141,20 +141,37 @@ dense_decode_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc,
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // last CTA of this (sequence, KV head): each warp merges its row; a lane owns 4 dims
+  // last CTA of this (sequence, KV head): each warp merges its row (lane t fetches (m, Z) of
+  // partials t, t + 32, ...; then every lane sums its 4 dims over the partials, 8 in flight)
   const float* rp = part + (size_t)row * S * kDensePart;
   float m_r = -CUDART_INF_F;
-  for (int s = 0; s < S; ++s)
-    if (__ldcg(rp + s * kDensePart + 1) > 0.f) m_r = fmaxf(m_r, __ldcg(rp + s * kDensePart));
+  for (int s = lane; s < S; s += 32) {
+    const float2 mz = __ldcg(reinterpret_cast<const float2*>(rp + (size_t)s * kDensePart));
+    if (mz.y > 0.f) m_r = fmaxf(m_r, mz.x);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m_r = fmaxf(m_r, __shfl_xor_sync(0xffffffffu, m_r, o));
   float Z_r = 0.f;
   float4 N_r = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < S; ++s) {
-    const float Zs = __ldcg(rp + s * kDensePart + 1);
-    const float a = safe_scale(__ldcg(rp + s * kDensePart), m_r, Zs);
-    const float* np = rp + s * kDensePart + 2 + 4 * lane;
-    Z_r = fmaf(Zs, a, Z_r);
-    N_r.x = fmaf(__ldcg(np), a, N_r.x); N_r.y = fmaf(__ldcg(np + 1), a, N_r.y);
-    N_r.z = fmaf(__ldcg(np + 2), a, N_r.z); N_r.w = fmaf(__ldcg(np + 3), a, N_r.w);
+  for (int s0 = 0; s0 < S; s0 += 8) {
+    float2 mz[8];
+    float4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      mz[u] = make_float2(0.f, 0.f);
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (s0 + u < S) {
+        mz[u] = __ldcg(reinterpret_cast<const float2*>(rp + (size_t)(s0 + u) * kDensePart));
+        v[u] = __ldcg(reinterpret_cast<const float4*>(rp + (size_t)(s0 + u) * kDensePart + 4) + lane);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const float a = safe_scale(mz[u].x, m_r, mz[u].y);
+      Z_r = fmaf(mz[u].y, a, Z_r);
+      N_r.x = fmaf(v[u].x, a, N_r.x); N_r.y = fmaf(v[u].y, a, N_r.y);
+      N_r.z = fmaf(v[u].z, a, N_r.z); N_r.w = fmaf(v[u].w, a, N_r.w);
+    }
   }
   const float inv = Z_r > 0.f ? 1.f / Z_r : 0.f;
   T* o = out + (size_t)row * kHeadDim + 4 * lane;

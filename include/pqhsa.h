@@ -28,7 +28,7 @@
  *   - v1 limits: head_dim == 128; pq_ncode == 256 (uint8 codes); pq_m in {8,16,32,64} with
  *     pq_m * pq_dsub == 128; n_list <= 4096 (and the per-CTA tables must fit shared memory,
  *     see PQHSA_ERR_UNSUPPORTED); max_seq_len % 4 == 0; page rows 16-byte aligned
- *     (strides multiples of 8 elements); n_sink == n_local == 0.
+ *     (strides multiples of 8 elements).
  */
 #ifndef PQHSA_H_
 #define PQHSA_H_
@@ -64,13 +64,18 @@ typedef struct {
   int32_t max_seq_len;        /* N_max: row stride of codes / list_ids / key_norms / scores */
   int32_t page_size;          /* tokens per KV page                                         */
   int32_t max_pages_per_seq;  /* row stride of block_table                                  */
-  int32_t n_sink;             /* |S| sink prefix (Sec. 3.2); must be 0 in v1                */
-  int32_t n_local;            /* |L| local window (Sec. 3.2); must be 0 in v1               */
+  int32_t n_sink;             /* sink prefix: S_b = first min(n_sink, N_b) tokens (Sec. 3.2) */
+  int32_t n_local;            /* local window: L_b = last min(n_local, N_b - |S_b|) tokens;  */
+                              /* R_b = the tokens between; S_b and L_b are attended exactly  */
+                              /* and take no part in the top-k or the background             */
   uint32_t budget_ppm;        /* rho in parts per million; k_b = ceil(|R_b| * ppm / 1e6),   */
                               /* computed in 64-bit integers on the device from seq_lens    */
   int32_t k_max;              /* row stride of sel_idx; >= ceil(max_seq_len * ppm / 1e6)    */
   float sm_scale;             /* 1/sqrt(d) (Eq. 1)                                          */
   int32_t dtype;              /* pqhsa_dtype of q, K, V and out                             */
+  int32_t exact_set_multiple; /* 0 or 1: off.  m > 1: |S_b| + |L_b| + k_b is rounded up to a  */
+                              /* multiple of m (App. A, budgets in whole pages), k_b <= |R_b|; */
+                              /* k_max must then cover the extra m - 1                        */
 } pqhsa_params;
 
 /* IVF-PQ index, one per (sequence, KV head) (Sec. 3.1).  Device pointers, read-only. */
@@ -126,24 +131,29 @@ int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index
                     float* lut, float* coarse, void* stream);
 
 /* Step 2 (Eq. 2 and the fused per-list reduction of Sec. 3.3).  seq_lens [B] int32.
- * Writes scores[b][h][i] = l~_i for i < seq_lens[b], and for every segment s of the row
- * (a contiguous token range scanned by one CTA; at most n_part per row, the count is a
- * function of seq_lens only) list_partials[b][h][s][0] = ref_s = max l~_i of the segment
- * and [1+j] = sum over the segment's members of list j of exp(l~_i - ref_s). */
+ * Writes scores[b][h][i] = l~_i for the tokens i of the indexed region R_b and -inf for the
+ * sink and window tokens (i < seq_lens[b]; they never compete in the top-k), and for every
+ * segment s of the row (a contiguous token range scanned by one CTA; at most n_part per row,
+ * the count is a function of seq_lens only) list_partials[b][h][s][0] = ref_s = max l~_i
+ * over the segment's tokens of R_b (-inf if it has none) and [1+j] = sum over the segment's
+ * members of list j inside R_b of exp(l~_i - ref_s). */
 int pqhsa_scan(const pqhsa_params* params, const pqhsa_index* index, const float* lut,
                const float* coarse, const int32_t* seq_lens, float* scores,
                float* list_partials, void* ws, size_t ws_bytes, void* stream);
 
 /* Step 3 (Eq. 3).  Exact top-k of every score row: sel_idx[b][h][0..k_b) = positions of the
- * k_b largest scores (order unspecified; equal scores: lower position first),
- * sel_count[b][h] = k_b, kth_score[b][h] = the k_b-th largest score (NaN if k_b == 0). */
+ * k_b largest scores among positions [0, seq_lens[b]) (order unspecified; equal scores:
+ * lower position first), sel_count[b][h] = k_b, kth_score[b][h] = the k_b-th largest score
+ * (NaN if k_b == 0).  k_b comes from |R_b| (see pqhsa_params); positions outside R_b are
+ * expected to hold -inf, as pqhsa_scan writes them, so that they rank last. */
 int pqhsa_select(const pqhsa_params* params, const float* scores, const int32_t* seq_lens,
                  int32_t* sel_idx, int32_t* sel_count, float* kth_score,
                  void* ws, size_t ws_bytes, void* stream);
 
-/* Step 4 (Eq. 4-5).  Gathers the selected K/V rows from the paged cache, replaces their
- * approximate logits by exact ones, takes the selected tokens' mass out of their lists'
- * sums, folds in the n_list mean-value terms and normalises once.
+/* Step 4 (Eq. 4-5).  Gathers the K/V rows of the exact set E_b = S_b u L_b u T (sinks, window,
+ * selected tokens) from the paged cache and attends them with exact logits, takes the
+ * selected tokens' approximate mass out of their lists' sums, folds in the n_list
+ * mean-value terms and normalises once.
  * out [B][H_q][d] in params->dtype; lse_or_null [B][H_q] = log of the normaliser. */
 int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
                         const pqhsa_index* index, const float* scores,

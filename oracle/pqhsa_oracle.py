@@ -209,7 +209,7 @@ def decode_head(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans
 def decode(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
            k_cache_flat, v_cache_flat, block_table, seq_lens, *, n_kv_heads, page_size,
            stride_page, stride_token, stride_head, budget_ppm, sm_scale,
-           n_sink=0, n_local=0, heads=None, batch_items=None):
+           n_sink=0, n_local=0, heads=None, batch_items=None, round_exact_set_to_page=0):
     """The whole operator: every (sequence, query head), reading the paged cache in
     place.  Array layouts are those of the C ABI (q [B,Hq,d]; centroids
     [B,Hkv,n_list,d]; codebooks [B,Hkv,M,n_code,dsub]; codes [B,Hkv,N_max,M];
@@ -232,5 +232,5 @@ def decode(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
             out[(b, h)] = decode_head(
                 q[b, h], centroids[b, g], codebooks[b, g], codes[b, g], list_ids[b, g],
                 None if key_norms is None else key_norms[b, g], list_vmeans[b, g],
-                keys, vals, n, budget_ppm, sm_scale, n_sink, n_local)
+                keys, vals, n, budget_ppm, sm_scale, n_sink, n_local, round_exact_set_to_page)
     return out

@@ -43,7 +43,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (p->batch <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->head_dim <= 0 ||
       p->n_list <= 0 || p->pq_m <= 0 || p->pq_dsub <= 0 || p->pq_ncode <= 0 ||
       p->max_seq_len <= 0 || p->page_size <= 0 || p->max_pages_per_seq <= 0 || p->k_max <= 0 ||
-      p->n_sink < 0 || p->n_local < 0)
+      p->n_sink < 0 || p->n_local < 0 || p->exact_set_multiple < 0)
     return PQHSA_ERR_INVALID_ARG;
   if (p->n_q_heads % p->n_kv_heads != 0) return PQHSA_ERR_INVALID_ARG;
   if (p->pq_m * p->pq_dsub != p->head_dim) return PQHSA_ERR_INVALID_ARG;
@@ -51,13 +51,14 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (p->dtype != PQHSA_F16 && p->dtype != PQHSA_BF16) return PQHSA_ERR_INVALID_ARG;
   if (!(p->sm_scale > 0.f)) return PQHSA_ERR_INVALID_ARG;
   if ((long long)p->max_pages_per_seq * p->page_size < p->max_seq_len) return PQHSA_ERR_INVALID_ARG;
-  const long long k_need = ((long long)p->max_seq_len * p->budget_ppm + 999999LL) / 1000000LL;
+  long long k_need = ((long long)p->max_seq_len * p->budget_ppm + 999999LL) / 1000000LL;
+  if (p->exact_set_multiple > 1) k_need += p->exact_set_multiple - 1;     // rounding slack
+  if (k_need > p->max_seq_len) k_need = p->max_seq_len;
   if (p->k_max < k_need) return PQHSA_ERR_INVALID_ARG;
 
   if (p->head_dim != kHeadDim || p->pq_ncode != kNCode) return PQHSA_ERR_UNSUPPORTED;
   if (p->pq_m != 8 && p->pq_m != 16 && p->pq_m != 32 && p->pq_m != 64) return PQHSA_ERR_UNSUPPORTED;
   if (p->n_list > 4096 || p->max_seq_len % 4 != 0) return PQHSA_ERR_UNSUPPORTED;
-  if (p->n_sink != 0 || p->n_local != 0) return PQHSA_ERR_UNSUPPORTED;
   const int G = p->n_q_heads / p->n_kv_heads;
   if (G > 16) return PQHSA_ERR_UNSUPPORTED;
 
@@ -67,7 +68,8 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.n_hg = (G + o.Gc - 1) / o.Gc;
   o.n_list = p->n_list; o.M = p->pq_m; o.dsub = p->pq_dsub;
   o.N_max = p->max_seq_len; o.page_size = p->page_size; o.max_pages = p->max_pages_per_seq;
-  o.k_max = p->k_max; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
+  o.k_max = p->k_max; o.n_sink = p->n_sink; o.n_local = p->n_local;
+  o.exact_multiple = p->exact_set_multiple; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
   o.num_sms = sm_count();
   o.scan_ctas = o.num_sms;
   o.upb = o.Hkv * o.n_hg;
@@ -101,9 +103,11 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   // attend kernel, split-K CTAs per row: about 512 selected tokens each, but enough CTAs to
   // fill the GPU when there are few rows (one wave of 4 resident CTAs per SM, background
   // CTAs included), as long as every CTA keeps at least 32 tokens
-  o.splits = ceil_div(o.k_max, 512);
+  const long long n_exact = (long long)o.k_max + (o.n_sink < o.N_max ? o.n_sink : o.N_max) +
+                            (o.n_local < o.N_max ? o.n_local : o.N_max);
+  o.splits = ceil_div(n_exact, 512);
   int fill = (4 * o.num_sms - o.B * o.upb * o.bg_splits) / o.rows;
-  const int max_fill = o.k_max / 32 > 0 ? o.k_max / 32 : 1;
+  const int max_fill = n_exact / 32 > 0 ? (int)(n_exact / 32) : 1;
   if (fill > max_fill) fill = max_fill;
   if (o.splits < fill) o.splits = fill;
   if (o.splits > 64) o.splits = 64;

@@ -77,6 +77,10 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   __syncthreads();
   float m = -CUDART_INF_F;
   for (int s = 0; s < nseg; ++s) m = fmaxf(m, s_scale[s]);
+  if (!(m > -CUDART_INF_F)) {            // no token of R in this row: no background at all
+    if (c == 0 && tid == 0) bg_max[row] = -CUDART_INF_F;
+    return;
+  }
   const float m2 = m * kLog2e;
   __syncthreads();
   if (tid < nseg) s_scale[tid] = fast_exp2(fmaf(s_scale[tid], kLog2e, -m2));
@@ -127,8 +131,9 @@ __global__ void __launch_bounds__(kAttendThreads, 4)
 attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
               long long stride_page, long long stride_token, long long stride_head,
               const int32_t* __restrict__ block_table, const int32_t* __restrict__ sel_idx,
-              const int32_t* __restrict__ sel_count, const float* __restrict__ bg_mass,
-              const float* __restrict__ bg_max, const float* __restrict__ vmeans,
+              const int32_t* __restrict__ sel_count, const int32_t* __restrict__ seq_lens,
+              const float* __restrict__ bg_mass, const float* __restrict__ bg_max,
+              const float* __restrict__ vmeans,
               float* __restrict__ split_part, uint32_t* __restrict__ tickets,
               T* __restrict__ out, float* __restrict__ lse) {
   constexpr int kWarps = kAttendThreads / 32;
@@ -216,14 +221,25 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   const int row = (int)blockIdx.x / S, split = (int)blockIdx.x % S;
   const int b = row / pl.Hq, h = row % pl.Hq, kv = h / pl.G;
   pdl_launch_dependents();
+  // the exact set E = T u S u L (Sec. 3.2), as one index space: the selected tokens first,
+  // then the sink prefix, then the local window
   const int cnt = sel_count[row];
-  const int tl = (int)((long long)split * cnt / S);
-  const int th = (int)((long long)(split + 1) * cnt / S);
+  const int n_seq = clamp_len(seq_lens[b], pl.N_max);
+  const Region rg = region_of(n_seq, pl.n_sink, pl.n_local);
+  const int n_s = rg.r_begin, n_exact = cnt + n_s + (n_seq - rg.r_end);
+  const int tl = (int)((long long)split * n_exact / S);
+  const int th = (int)((long long)(split + 1) * n_exact / S);
   const int per_warp = (th - tl + kWarps - 1) / kWarps;
   const int wl = min(th, tl + warp * per_warp), wh = min(th, wl + per_warp);
   const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
   const int32_t* bt = block_table + (size_t)b * pl.max_pages;
-  int my_pos = (wl + lane < wh) ? sel[wl + lane] : -1;
+  auto pos_of = [&](int t) -> int {        // position of item t of E, -1 past the warp's slice
+    if (t >= wh) return -1;
+    if (t < cnt) return sel[t];
+    const int u = t - cnt;
+    return u < n_s ? u : rg.r_end + (u - n_s);
+  };
+  int my_pos = pos_of(wl + lane);
 
   const int gi = lane >> 3, gl = lane & 7;      // lane group (4 per warp) and lane in group
   float qf[16];
@@ -250,7 +266,7 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
     if (my_pos >= 0)
       off = (long long)my_page * stride_page + (long long)(my_pos % pl.page_size) * stride_token +
             (long long)kv * stride_head;
-    const int nxt_pos = (base + 32 + lane < wh) ? sel[base + 32 + lane] : -1;
+    const int nxt_pos = pos_of(base + 32 + lane);
     int nxt_page = 0;
     const int nb = min(32, wh - base);
     for (int j0 = 0; j0 < nb; j0 += 4 * U) {
@@ -376,14 +392,15 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
                       static_cast<const __half*>(q), static_cast<const __half*>(kv.k_cache),
                       static_cast<const __half*>(kv.v_cache), (long long)kv.stride_page,
                       (long long)kv.stride_token, (long long)kv.stride_head, kv.block_table,
-                      sel_idx, sel_count, bg_mass, bg_max, ix.list_vmeans, split_part, tickets,
+                      sel_idx, sel_count, seq_lens, bg_mass, bg_max, ix.list_vmeans, split_part,
+                      tickets,
                       static_cast<__half*>(out), lse);
   return launch_pdl(attend_kernel<__nv_bfloat16, 4>, grid, dim3(kAttendThreads), 0, st, pl,
                     static_cast<const __nv_bfloat16*>(q),
                     static_cast<const __nv_bfloat16*>(kv.k_cache),
                     static_cast<const __nv_bfloat16*>(kv.v_cache), (long long)kv.stride_page,
                     (long long)kv.stride_token, (long long)kv.stride_head, kv.block_table, sel_idx,
-                    sel_count, bg_mass, bg_max, ix.list_vmeans, split_part, tickets,
+                    sel_count, seq_lens, bg_mass, bg_max, ix.list_vmeans, split_part, tickets,
                     static_cast<__nv_bfloat16*>(out), lse);
 }
 

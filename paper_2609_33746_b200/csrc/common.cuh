@@ -32,6 +32,8 @@ struct Plan {
   int n_list, M, dsub;
   int N_max, page_size, max_pages;
   int k_max;
+  int n_sink, n_local;               // |S| and |L| of Sec. 3.2 (upper bounds: clipped per sequence)
+  int exact_multiple;                // > 1: |S| + |L| + k is rounded up to this multiple (App. A)
   uint32_t ppm;
   float sm_scale;
   int dtype;
@@ -90,6 +92,32 @@ __device__ __forceinline__ int budget_k(int n, uint32_t ppm) {
 
 __device__ __forceinline__ int clamp_len(int n, int n_max) {
   return n < 0 ? 0 : (n > n_max ? n_max : n);
+}
+
+// Position partition of a sequence of n tokens (Sec. 3.2): sink prefix S = [0, r_begin),
+// indexed region R = [r_begin, r_end), local window L = [r_end, n).
+struct Region {
+  int r_begin, r_end;
+};
+__device__ __forceinline__ Region region_of(int n, int n_sink, int n_local) {
+  Region r;
+  r.r_begin = n_sink < n ? n_sink : n;
+  r.r_end = n - n_local > r.r_begin ? n - n_local : r.r_begin;
+  return r;
+}
+// k of Eq. 3 for a sequence of n tokens: ceil(rho |R|); with exact_multiple > 1 the size of
+// the exact set |S| + |L| + k is rounded up to that multiple first (never beyond |R|).
+__device__ __forceinline__ int region_budget(int n, int n_sink, int n_local, uint32_t ppm,
+                                             int exact_multiple) {
+  const Region r = region_of(n, n_sink, n_local);
+  const int n_r = r.r_end - r.r_begin;
+  int k = budget_k(n_r, ppm);
+  if (exact_multiple > 1) {
+    const long long fixed = n - n_r;
+    const long long total = (fixed + k + exact_multiple - 1) / exact_multiple * exact_multiple;
+    k = (int)(total - fixed < n_r ? total - fixed : n_r);
+  }
+  return k;
 }
 
 // The scan walks one global sequence of 32-token tiles: sequence-major, then the

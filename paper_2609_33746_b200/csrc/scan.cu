@@ -264,6 +264,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     const int cnt = (int)min((long long)(tb - t0), hi - lo);
     const int slot = c - split_cta_of(sp, base + (long long)w * tb);
     const int Nb = clamp_len(seq_lens[b], N_max);
+    const Region rg = region_of(Nb, pl.n_sink, pl.n_local);   // only R enters top-k and sums
     const int kv = w / pl.n_hg, hg = w % pl.n_hg;
     const size_t ukv = (size_t)b * pl.Hkv + kv;
     const size_t unit = ukv * pl.n_hg + hg;
@@ -314,6 +315,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
       __syncwarp();      // the copies of all lanes for tile t have landed
       const int i = t * kTile + lane;
       const bool valid = have && i < Nb;
+      const bool in_r = valid && i >= rg.r_begin && i < rg.r_end;
       float sc[GC];
 #pragma unroll
       for (int g = 0; g < GC; ++g) sc[g] = -CUDART_INF_F;
@@ -352,10 +354,12 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         if (pl.coarse_in_smem) load_vec<GC>(co, s_coarse + cur.lid * GC);
         else load_vec<GC>(co, g_coarse + cur.lid * GC);
         if (valid) {
+          // sink and window tokens are attended exactly: their score is -inf, so that the
+          // top-k never picks them and they add nothing to the list sums
 #pragma unroll
           for (int g = 0; g < GC; ++g) {
             if (g < n_heads) {
-              sc[g] = cur.norm * (co[g] + accf[g]);
+              if (in_r) sc[g] = cur.norm * (co[g] + accf[g]);
               scores[(size_t)(row0 + g) * N_max + i] = sc[g];
               mx[g] = fmaxf(mx[g], sc[g]);
             }
@@ -381,7 +385,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         if (tid < GC) s_ref[tid] = ref2[tid];
         first = false;
       }
-      if (valid) {
+      if (in_r) {
         float x[GC], xm = -CUDART_INF_F;
 #pragma unroll
         for (int g = 0; g < GC; ++g) {
@@ -435,7 +439,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         for (int g = 0; g < GC; ++g) {
           if (g < n_heads) {
             const float s = __ldcg(scores + (size_t)(row0 + g) * N_max + i);
-            const float x = fmaf(s, kLog2e, -s_ref[g]);
+            const float x = fmaf(s, kLog2e, -s_ref[g]);     // -inf or NaN outside R
             if (x > kNegligibleLog2) atomicAdd(&s_sums[g * n_list + lid], fast_exp2(x));
           }
         }
@@ -445,7 +449,8 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     // flush: header = segment maximum, sums re-based from the reference to that maximum
     for (int idx = tid; idx < n_heads * (n_list + 1); idx += kScanThreads) {
       const int g = idx / (n_list + 1), j = idx - g * (n_list + 1);
-      const float rescale = fast_exp2(s_ref[g] - s_max[g] * kLog2e);
+      // a segment without any token of R has maximum -inf and empty sums
+      const float rescale = s_max[g] > -CUDART_INF_F ? fast_exp2(s_ref[g] - s_max[g] * kLog2e) : 0.f;
       const float v = (j == 0) ? s_max[g] : s_sums[g * n_list + j - 1] * rescale;
       partials[((size_t)(row0 + g) * pl.n_part + slot) * (n_list + 1) + j] = v;
     }

@@ -174,12 +174,13 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
   pdl_wait();
   pdl_launch_dependents();
   const int n = clamp_len(seq_lens[b], pl.N_max);
-  const int k = budget_k(n, pl.ppm);
+  const int k = region_budget(n, pl.n_sink, pl.n_local, pl.ppm, pl.exact_multiple);
+  const Region rg = region_of(n, pl.n_sink, pl.n_local);
   float lo = -CUDART_INF_F, hi = CUDART_INF_F;     // default: every score is a candidate
   if (k == 0) {
     if (tid == 0) { sel_count[row] = 0; kth[row] = CUDART_NAN_F; }
-  } else if (k == n) {
-    hi = -CUDART_INF_F;                            // every finite score is a winner
+  } else if (k == rg.r_end - rg.r_begin) {
+    hi = -CUDART_INF_F;                            // all of R: every score above -inf is a winner
   } else if (n > kSelChunk) {
     // 1024 aligned groups of 4 consecutive scores; group g sits in the g-th of 1024 equal
     // strides of the row at a hashed offset (reads 16 bytes per touched 32-byte sector)

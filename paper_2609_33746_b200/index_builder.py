@@ -146,10 +146,14 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
             cb = _batched_pq_kmeans(res_fit.view(-1, M, dsub), nc, cfg.kmeans_iters, gen)
             res = (u - c[ids]).view(n, M, dsub).permute(1, 0, 2).contiguous()
             codes = _pq_encode(res, cb)                           # [M, n]
+            # list value means over the members inside the indexed region R (Sec. 3.2): sink
+            # and window tokens are attended exactly and belong to no list's background
+            r0 = min(cfg.n_sink, n)
+            r1 = max(r0, n - cfg.n_local)
             vsum = torch.zeros((nl, d), dtype=torch.float64, device=dev).index_add_(
-                0, ids, v.double())
+                0, ids[r0:r1], v[r0:r1].double())
             cnt = torch.zeros(nl, dtype=torch.float64, device=dev).index_add_(
-                0, ids, torch.ones(n, dtype=torch.float64, device=dev))
+                0, ids[r0:r1], torch.ones(r1 - r0, dtype=torch.float64, device=dev))
             vmean = torch.where(cnt[:, None] > 0, vsum / cnt.clamp(min=1)[:, None],
                                 torch.zeros_like(vsum))
             out.centroids[b, g] = c

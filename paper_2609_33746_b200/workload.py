@@ -52,6 +52,9 @@ class DecodeConfig:
     kv_layout: str = "split"             # "split": K and V separate [page][tok][head][d]
                                          # "interleaved": one buffer [page][head][tok][2d]
     fit_sample: int = 0                  # >0: fit centroids/codebooks on this many tokens
+    n_sink: int = 0                      # |S|: first tokens attended exactly (Sec. 3.2)
+    n_local: int = 0                     # |L|: most recent tokens attended exactly
+    exact_set_multiple: int = 0          # >1: |S|+|L|+k rounded up to this multiple (App. A)
 
     @property
     def group(self) -> int:

@@ -60,7 +60,9 @@ def run_oracle(inp, idx, budget_ppm=None, heads=None, batch_items=None, arrays=N
                     page_size=cfg.page_size, stride_page=inp.stride_page,
                     stride_token=inp.stride_token, stride_head=inp.stride_head,
                     budget_ppm=cfg.budget_ppm if budget_ppm is None else budget_ppm,
-                    sm_scale=1.0 / math.sqrt(cfg.head_dim), heads=heads, batch_items=batch_items)
+                    sm_scale=1.0 / math.sqrt(cfg.head_dim), heads=heads, batch_items=batch_items,
+                    n_sink=cfg.n_sink, n_local=cfg.n_local,
+                    round_exact_set_to_page=cfg.exact_set_multiple if cfg.exact_set_multiple > 1 else 0)
 
 
 def selection_matches(gpu_sel, ref, tol=1e-3):

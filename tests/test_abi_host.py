@@ -68,8 +68,9 @@ def test_group_of_eight_is_two_head_groups_and_padded_groups():
 
 
 @pytest.mark.parametrize("kw,status", [
-    (dict(n_sink=4), pqhsa.ERR_UNSUPPORTED),             # sinks / window: not on the GPU path yet
-    (dict(n_local=128), pqhsa.ERR_UNSUPPORTED),
+    (dict(n_sink=-1), pqhsa.ERR_INVALID_ARG),
+    (dict(n_local=-5), pqhsa.ERR_INVALID_ARG),
+    (dict(exact_set_multiple=16, k_max=1311), pqhsa.ERR_INVALID_ARG),   # no room for the rounding
     (dict(head_dim=64, pq_m=16), pqhsa.ERR_UNSUPPORTED),
     (dict(pq_m=4), pqhsa.ERR_UNSUPPORTED),
     (dict(n_list=8192), pqhsa.ERR_UNSUPPORTED),

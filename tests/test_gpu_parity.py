@@ -60,6 +60,14 @@ CASES = {
     "norm_jump": small("jump", seq_lens=(40000,), n_q_heads=4, n_kv_heads=1, kmeans_iters=1),
     "odd_list_count": small("odd", seq_lens=(1000,), n_list=37, n_q_heads=2, n_kv_heads=2,
                             kmeans_iters=1),
+    # the paper's own partition: 4 sinks and a 128-token window attended exactly (Sec. 3.2)
+    "sinks_and_window": small("sw", seq_lens=(5000,), n_sink=4, n_local=128),
+    # ... with the exact set rounded up to whole pages of 16 (App. A), ragged batch whose
+    # short sequences are all sink / all window / have an empty indexed region
+    "sinks_window_pages_ragged": small("swr", batch=5, seq_lens=(3000, 3, 100, 132, 9000),
+                                       n_q_heads=4, n_kv_heads=1, n_sink=4, n_local=128,
+                                       exact_set_multiple=16),
+    "window_only_g8": small("w8", n_q_heads=16, n_kv_heads=2, seq_lens=(2500,), n_local=64),
 }
 
 
@@ -132,10 +140,15 @@ def test_stage_scan_scores_and_list_sums(key):
     parts = op.list_partials.view(cfg.batch, cfg.n_q_heads, n_part, cfg.n_list + 1).cpu().double().numpy()
     for (b, h), r in ref.items():
         n = int(arrays["seq_lens"][b])
-        got, want = scores[b, h, :n], r["approx"]
+        R = r["R"]                                      # indexed region: positions r0 .. r1-1
+        r0, r1 = (int(R[0]), int(R[-1]) + 1) if len(R) else (0, 0)
+        got, want = scores[b, h, r0:r1], r["approx"]
         assert np.all(np.abs(got - want) <= LOGIT_RTOL * np.maximum(np.abs(want), 1.0)), \
             f"logits differ at {(b, h)}: {np.abs(got - want).max()}"
-        if n == 0:
+        # sink and window positions never compete in the top-k
+        outside = np.concatenate([scores[b, h, :r0], scores[b, h, r1:n]]) if len(R) else scores[b, h, :n]
+        assert np.all(np.isneginf(outside))
+        if len(R) == 0:
             continue
         # per-list exp-sums over ALL members, merged over the scan's segments
         p = parts[b, h]
@@ -144,7 +157,7 @@ def test_stage_scan_scores_and_list_sums(key):
         m = p[used, 0].max()
         assert abs(m - want.max()) <= LOGIT_RTOL * max(1.0, abs(want.max()))
         tot = (p[used, 1:] * np.exp(p[used, 0] - m)[:, None]).sum(axis=0)
-        lists = arrays["list_ids"][b, h // cfg.group, :n].astype(np.int64)
+        lists = arrays["list_ids"][b, h // cfg.group, r0:r1].astype(np.int64)
         want_tot = np.bincount(lists, weights=np.exp(want - want.max()), minlength=cfg.n_list)
         assert np.abs(tot - want_tot).max() <= 2e-4 * want_tot.sum()
 
@@ -296,7 +309,7 @@ def test_rows_that_defeat_the_sample_fall_back_to_the_exact_path():
 def test_invalid_arguments_launch_nothing():
     inp, idx, arrays, ref, op = get_case("c1")
     bad = pqhsa.Params.from_buffer_copy(op.params)
-    bad.n_sink = 4
+    bad.n_list = 8192
     with pytest.raises(pqhsa.PqhsaError) as e:
         pqhsa.decode(bad, op.q, op.index, op.kv, op.seq_lens, op.out, op.ws)
     assert e.value.status == pqhsa.ERR_UNSUPPORTED
@@ -371,3 +384,35 @@ def test_dense_comparator_is_textbook_attention(key):
                               cfg.page_size, inp.stride_page, inp.stride_token, inp.stride_head)
             want = softmax(K @ arrays["q"][b, h] / math.sqrt(128.0)) @ V
             assert np.all(np.abs(got[b, h] - want) <= out_tolerance(want, cfg.dtype))
+
+
+def test_paper_budgets_on_the_device():
+    """App. A prints the exact-set sizes of the 128K setting (4 sinks, 128-token window, pages
+    of 16): the device's integer budget arithmetic must land on the same totals, and the
+    selected positions must stay inside the indexed region."""
+    import pathlib
+    rows = [l.split() for l in (pathlib.Path(__file__).parent / "golden" / "paper_budgets.txt")
+            .read_text().splitlines() if l.strip() and not l.startswith("#")]
+    for seq_len, n_sink, n_local, ppm, page, tokens in (tuple(map(int, r)) for r in rows):
+        p = pqhsa.make_params(batch=1, n_q_heads=2, n_kv_heads=2, n_list=64, pq_m=32,
+                              max_seq_len=seq_len, max_pages_per_seq=seq_len // 16,
+                              budget_ppm=ppm, dtype="bf16", n_sink=n_sink, n_local=n_local,
+                              exact_set_multiple=page)
+        g = torch.Generator(device="cuda").manual_seed(5)
+        scores = torch.randn((2, seq_len), generator=g, device="cuda")
+        scores[:, :n_sink] = float("-inf")                    # as pqhsa_scan leaves S and L
+        scores[:, seq_len - n_local:] = float("-inf")
+        lens = torch.tensor([seq_len], dtype=torch.int32, device="cuda")
+        sel = torch.full((2, p.k_max), -1, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(2, dtype=torch.int32, device="cuda")
+        kth = torch.zeros(2, dtype=torch.float32, device="cuda")
+        ws = torch.empty(pqhsa.workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        pqhsa.select(p, scores, lens, sel, cnt, kth, ws)
+        torch.cuda.synchronize()
+        k = tokens - n_sink - n_local
+        assert cnt.tolist() == [k, k]
+        for h in range(2):
+            got = sel[h, :k].cpu().numpy()
+            assert got.min() >= n_sink and got.max() < seq_len - n_local
+            want = O.select_topk(scores[h, n_sink:seq_len - n_local].cpu().double().numpy(), k) + n_sink
+            assert sorted(got.tolist()) == want.tolist()

@@ -204,13 +204,17 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
       part[4 + tid] = N_c;
       if (tid == 0) { part[0] = bg_max[row0 + g] * kLog2e; part[1] = Z_c; }
     }
-    __threadfence();
+    // one ticket per row of the group (see cta_arrived_last for the fences)
     __syncthreads();
-    if (tid < n_heads) s_last[tid] = (atomicAdd(&tickets[row0 + tid], 1u) == (uint32_t)(n_part - 1));
+    if (tid < n_heads) {
+      __threadfence();
+      const bool last = atomicAdd(&tickets[row0 + tid], 1u) == (uint32_t)(n_part - 1);
+      if (last) __threadfence();
+      s_last[tid] = last ? 1 : 0;
+    }
     __syncthreads();
     for (int g = 0; g < n_heads; ++g) {
       if (!s_last[g]) continue;
-      __threadfence();
       merge_row(split_part + (size_t)(row0 + g) * n_part * kPartStride, n_part, row0 + g, tid,
                 s_N, s_aux, out, lse);
     }
@@ -362,12 +366,7 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   float* part = split_part + ((size_t)row * n_part + split) * kPartStride;
   part[4 + tid] = N_c;
   if (tid == 0) { part[0] = m_c; part[1] = Z_c; }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last[0] = (atomicAdd(&tickets[row], 1u) == (uint32_t)(n_part - 1));
-  __syncthreads();
-  if (!s_last[0]) return;
-  __threadfence();
+  if (!cta_arrived_last(&tickets[row], (uint32_t)n_part, &s_last[0])) return;
   merge_row(split_part + (size_t)row * n_part * kPartStride, n_part, row, tid, s_N, s_aux, out, lse);
 }
 

@@ -165,6 +165,24 @@ __device__ __forceinline__ void pdl_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Last-arrival ticket among the CTAs that share `counter`.  Every thread of the CTA calls it
+// after the CTA's global writes; it returns true, to all threads, in the CTA that arrived
+// last, which may then read what the others wrote.  One thread fences for the whole CTA
+// (fences are cumulative): the first barrier orders the CTA's writes before that thread's
+// fence and draw, the second orders its draw and fence before the CTA's reads.  Nobody waits.
+__device__ __forceinline__ bool cta_arrived_last(uint32_t* counter, uint32_t n_arrivals,
+                                                 int* s_flag) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const bool last = atomicAdd(counter, 1u) == n_arrivals - 1u;
+    if (last) __threadfence();
+    *s_flag = last ? 1 : 0;
+  }
+  __syncthreads();
+  return *s_flag != 0;
+}
+
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));

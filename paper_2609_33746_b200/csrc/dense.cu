@@ -135,12 +135,7 @@ dense_decode_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc,
     }
     if (gl == 0) { pr[0] = st.m; pr[1] = st.Z; }
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&tickets[b * pl.Hkv + kv], 1u) == (uint32_t)(S - 1));
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
+  if (!cta_arrived_last(&tickets[b * pl.Hkv + kv], (uint32_t)S, &s_last)) return;
   // last CTA of this (sequence, KV head): each warp merges its row (lane t fetches (m, Z) of
   // partials t, t + 32, ...; then every lane sums its 4 dims over the partials, 8 in flight)
   const float* rp = part + (size_t)row * S * kDensePart;

@@ -40,11 +40,21 @@ __device__ void find_digit(const uint32_t* hist, int nbins, int k, int* s_scan, 
   const int hi = nbins - tid * per;
   uint32_t mine[8];
   uint32_t local = 0;
+  if (per == 8 && hi >= 8) {
+    // two 16-byte reads instead of eight 4-byte reads 32 bytes apart (8-way bank conflicts)
+    const uint4 v0 = *reinterpret_cast<const uint4*>(hist + hi - 8);
+    const uint4 v1 = *reinterpret_cast<const uint4*>(hist + hi - 4);
+    mine[0] = v1.w; mine[1] = v1.z; mine[2] = v1.y; mine[3] = v1.x;
+    mine[4] = v0.w; mine[5] = v0.z; mine[6] = v0.y; mine[7] = v0.x;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int d = hi - 1 - j;
-    mine[j] = (j < per && d >= 0) ? hist[d] : 0u;
-    local += mine[j];
+    for (int j = 0; j < 8; ++j) local += mine[j];
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int d = hi - 1 - j;
+      mine[j] = (j < per && d >= 0) ? hist[d] : 0u;
+      local += mine[j];
+    }
   }
   if (tid == 0) { s_scan[32] = 0; s_scan[33] = 0; }
   uint32_t inc = local;
@@ -167,7 +177,8 @@ __global__ void __launch_bounds__(kSelThreads)
 sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __restrict__ seq_lens,
                   int32_t* __restrict__ rowstate, int32_t* __restrict__ sel_count,
                   float* __restrict__ kth) {
-  __shared__ uint32_t s_hist[kHistBins], s_hist_b[kHistBins];
+  __shared__ __align__(16) uint32_t s_hist[kHistBins];
+  __shared__ __align__(16) uint32_t s_hist_b[kHistBins];
   __shared__ int s_scan[34];
   const int row = blockIdx.x, tid = threadIdx.x;
   const int b = row / pl.Hq;
@@ -440,12 +451,7 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
     }
     __syncwarp();
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(&counters[row * 4 + 1], 1u) == gridDim.x - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
+  if (!cta_arrived_last(&counters[row * 4 + 1], gridDim.x, &s_last)) return;
 
   // ---- last CTA of the row: check the bracket by counting, then select among the candidates
   const int W = (int)__ldcg(n_out), C = (int)__ldcg(n_cand);

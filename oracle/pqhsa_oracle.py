@@ -18,6 +18,8 @@ re-ordering:
     O7  common shift m_0, e_i on E, e~_i on B = R \\ T                    (Sec. 3.2)
     O8  per-list background mass M_j, Z^_B, N^_B with the stored means   (Eq. 4)
     O9  y^ = (N_E + N^_B) / (Z_E + Z^_B)                                 (Eq. 5)
+    O10 index maintenance: new tokens encoded into the existing lists,  (Sec. 3.3, first paragraph;
+        list means refreshed, no re-clustering                           Sec. 3.1 for the encoding)
 
 Readings where the paper is silent (each also listed in the design doc):
   * top-k ties: stable, the lower position wins;
@@ -25,15 +27,20 @@ Readings where the paper is silent (each also listed in the design doc):
   * u_q = 0 when r_q = 0;
   * the list mean that multiplies M_j is the stored mean over all members of the
     list, selected ones included (Sec. 3.2, last paragraph);
-  * an empty list contributes zero (text after Eq. 4).
+  * an empty list contributes zero (text after Eq. 4);
+  * index maintenance: a new key goes to the list whose centroid is nearest to its direction
+    in squared Euclidean distance (the assignment rule of k-means, the lower index on ties),
+    each sub-vector of the residual to its nearest codeword likewise, a zero key has
+    direction 0, and the refreshed list mean is the mean over old and new members.
 
 Pins (tests/test_oracle_pins.py): brute-force loops on tiny inputs, the ADC sum
 against a dense dot product with the reconstructed key, rho = 1 against textbook
 softmax attention, the exact-reconstruction / constant-value-per-list case against
 textbook attention at any budget, a hand-computed closed form, mass conservation,
 shift and permutation invariance, the budgets the paper prints (1,456 and 2,752
-tokens at 131,072), and top-k against a full sort.  No function here is
-"parity unpinned".
+tokens at 131,072), and top-k against a full sort; for O10 scalar-loop brute force, the
+from-scratch mean of all members, a key on a centroid, and one update against two.  No
+function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -234,3 +241,60 @@ def decode(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
                 None if key_norms is None else key_norms[b, g], list_vmeans[b, g],
                 keys, vals, n, budget_ppm, sm_scale, n_sink, n_local, round_exact_set_to_page)
     return out
+
+
+# --------------------------------------------------------------------------- O10
+def encode_keys(keys: np.ndarray, centroids: np.ndarray, codebooks: np.ndarray):
+    """Direction-norm residual IVF-PQ encoding of keys [n, d] against fixed centroids
+    [n_list, d] and codebooks [M, n_code, dsub] (Sec. 3.1): r_i = |k_i|, u_i = k_i / r_i,
+    a_i = argmin_j |u_i - c_j|^2, z_im = argmin_z |(u_i - c_{a_i})^(m) - p_{m,z}|^2.
+    Returns (norms [n], list_ids [n], codes [n, M], d_coarse [n, n_list], d_pq [n, M, n_code]);
+    the two distance arrays let a test see how close a decision was."""
+    keys = np.asarray(keys, dtype=np.float64)
+    c = np.asarray(centroids, dtype=np.float64)
+    cb = np.asarray(codebooks, dtype=np.float64)
+    n, d = keys.shape
+    M, n_code, dsub = cb.shape
+    r = np.sqrt((keys * keys).sum(axis=1))
+    u = np.zeros_like(keys)
+    nz = r > 0
+    u[nz] = keys[nz] / r[nz, None]
+    d_coarse = ((u[:, None, :] - c[None, :, :]) ** 2).sum(axis=2)            # [n, n_list]
+    a = d_coarse.argmin(axis=1)                                              # first minimum
+    e = (u - c[a]).reshape(n, M, dsub)
+    d_pq = ((e[:, :, None, :] - cb[None, :, :, :]) ** 2).sum(axis=3)         # [n, M, n_code]
+    z = d_pq.argmin(axis=2)
+    return r, a, z, d_coarse, d_pq
+
+
+def index_update(centroids, codebooks, codes, list_ids, key_norms, list_vmeans, list_counts,
+                 new_keys, new_vals, first_pos: int):
+    """Index maintenance for one (sequence, KV head) (Sec. 3.3): the tokens at positions
+    first_pos, first_pos + 1, ... are encoded into the existing lists (no re-clustering),
+    and every list's value mean becomes the mean over its old and new members:
+    vbar_j <- (n_j vbar_j + sum of the new members' values) / (n_j + new_j).
+    Returns updated copies (codes, list_ids, key_norms, list_vmeans, list_counts) and the
+    distance arrays of encode_keys."""
+    new_vals = np.asarray(new_vals, dtype=np.float64)
+    r, a, z, d_coarse, d_pq = encode_keys(new_keys, centroids, codebooks)
+    n_new = len(r)
+    codes = np.array(codes, copy=True)
+    list_ids = np.array(list_ids, copy=True)
+    key_norms = np.array(key_norms, dtype=np.float64, copy=True)
+    vmeans = np.array(list_vmeans, dtype=np.float64, copy=True)
+    counts = np.array(list_counts, dtype=np.int64, copy=True)
+    pos = first_pos + np.arange(n_new)
+    codes[pos] = z.astype(codes.dtype)
+    list_ids[pos] = a.astype(list_ids.dtype)
+    key_norms[pos] = r
+    n_list = vmeans.shape[0]
+    added = np.bincount(a, minlength=n_list)
+    vsum = np.zeros_like(vmeans)
+    np.add.at(vsum, a, new_vals)
+    touched = added > 0
+    vmeans[touched] = (counts[touched, None] * vmeans[touched] + vsum[touched]) / \
+                      (counts[touched] + added[touched])[:, None]
+    counts = counts + added
+    return dict(codes=codes, list_ids=list_ids, key_norms=key_norms, list_vmeans=vmeans,
+                list_counts=counts, d_coarse=d_coarse, d_pq=d_pq)
+

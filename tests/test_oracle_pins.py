@@ -299,3 +299,101 @@ def test_gather_rows_two_layouts_and_flat_are_identical():
         vb = O.gather_rows(inter.ravel()[d:], table, pos, h, d, P, H * P * 2 * d, 2 * d,
                            P * 2 * d)
         assert np.array_equal(va, V[pos, h].astype(np.float64)) and np.array_equal(va, vb)
+
+
+# ----------------------------------------------------------------------------- O10 index maintenance
+def _tiny_index(rng, n_list=3, d=4, M=2, n_code=4, n_old=7):
+    centroids = rng.normal(size=(n_list, d))
+    codebooks = rng.normal(size=(M, n_code, d // M)) * 0.3
+    old_ids = rng.integers(0, n_list, size=n_old)
+    old_vals = rng.normal(size=(n_old, d))
+    vmeans = np.zeros((n_list, d))
+    counts = np.bincount(old_ids, minlength=n_list)
+    for j in range(n_list):
+        if counts[j]:
+            vmeans[j] = old_vals[old_ids == j].mean(axis=0)
+    N = n_old + 8
+    codes = np.zeros((N, M), dtype=np.uint8)
+    ids = np.zeros(N, dtype=np.uint16)
+    ids[:n_old] = old_ids
+    norms = np.zeros(N)
+    return centroids, codebooks, codes, ids, norms, vmeans, counts, old_ids, old_vals
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_index_update_brute_force_and_from_scratch_means(seed):
+    """Scalar loops for the assignment and the codes; the refreshed means against the mean of
+    all members computed from scratch."""
+    rng = np.random.default_rng(seed)
+    c, cb, codes, ids, norms, vmeans, counts, old_ids, old_vals = _tiny_index(rng)
+    n_old, n_new = len(old_ids), 5
+    keys = rng.normal(size=(n_new, 4)) * 2.0
+    vals = rng.normal(size=(n_new, 4))
+    out = O.index_update(c, cb, codes, ids, norms, vmeans, counts, keys, vals, first_pos=n_old)
+    M, n_code, dsub = cb.shape
+    for t in range(n_new):
+        r = math.sqrt(sum(x * x for x in keys[t]))
+        u = [x / r for x in keys[t]]
+        best, best_j = None, None
+        for j in range(len(c)):
+            dist = sum((u[i] - c[j][i]) ** 2 for i in range(4))
+            if best is None or dist < best:
+                best, best_j = dist, j
+        assert out["list_ids"][n_old + t] == best_j
+        assert abs(out["key_norms"][n_old + t] - r) < 1e-12
+        for m in range(M):
+            e = [u[m * dsub + i] - c[best_j][m * dsub + i] for i in range(dsub)]
+            bz, bd = None, None
+            for z in range(n_code):
+                dist = sum((e[i] - cb[m][z][i]) ** 2 for i in range(dsub))
+                if bd is None or dist < bd:
+                    bd, bz = dist, z
+            assert out["codes"][n_old + t, m] == bz
+    all_ids = np.concatenate([old_ids, out["list_ids"][n_old:n_old + n_new].astype(np.int64)])
+    all_vals = np.concatenate([old_vals, vals])
+    for j in range(len(c)):
+        members = all_vals[all_ids == j]
+        assert out["list_counts"][j] == len(members)
+        if len(members):
+            np.testing.assert_allclose(out["list_vmeans"][j], members.mean(axis=0), atol=1e-12)
+    # nothing outside the new positions moved
+    assert np.array_equal(out["codes"][:n_old], codes[:n_old])
+    assert np.array_equal(out["list_ids"][:n_old], ids[:n_old])
+
+
+def test_index_update_key_on_a_centroid_has_zero_residual():
+    """Orthonormal centroids: a key 3 e_j has norm 3, lands in list j, and its residual is 0,
+    so every sub-vector takes the zero codeword."""
+    c = np.eye(4)
+    cb = np.random.default_rng(3).normal(size=(2, 6, 2))
+    cb[:, 5, :] = 0.0
+    codes = np.zeros((4, 2), dtype=np.uint8)
+    out = O.index_update(c, cb, codes, np.zeros(4, dtype=np.uint16), np.zeros(4),
+                         np.zeros((4, 4)), np.zeros(4, dtype=np.int64),
+                         new_keys=3.0 * np.eye(4)[[2, 0]], new_vals=np.ones((2, 4)), first_pos=1)
+    assert out["list_ids"][1:3].tolist() == [2, 0]
+    assert out["key_norms"][1:3].tolist() == [3.0, 3.0]
+    assert out["codes"][1:3].tolist() == [[5, 5], [5, 5]]
+    assert out["list_counts"].tolist() == [1, 0, 1, 0]
+    np.testing.assert_array_equal(out["list_vmeans"][[0, 2]], np.ones((2, 4)))
+    # a zero key: direction 0, norm 0, nearest centroid by the same rule (all at distance 1: list 0)
+    out0 = O.index_update(c, cb, codes, np.zeros(4, dtype=np.uint16), np.zeros(4),
+                          np.zeros((4, 4)), np.zeros(4, dtype=np.int64),
+                          new_keys=np.zeros((1, 4)), new_vals=np.ones((1, 4)), first_pos=0)
+    assert out0["key_norms"][0] == 0.0 and out0["list_ids"][0] == 0
+
+
+def test_index_update_in_two_steps_equals_one_step():
+    rng = np.random.default_rng(9)
+    c, cb, codes, ids, norms, vmeans, counts, old_ids, old_vals = _tiny_index(rng, n_list=4)
+    n_old = len(old_ids)
+    keys = rng.normal(size=(8, 4))
+    vals = rng.normal(size=(8, 4))
+    one = O.index_update(c, cb, codes, ids, norms, vmeans, counts, keys, vals, first_pos=n_old)
+    a = O.index_update(c, cb, codes, ids, norms, vmeans, counts, keys[:3], vals[:3], first_pos=n_old)
+    b = O.index_update(c, cb, a["codes"], a["list_ids"], a["key_norms"], a["list_vmeans"],
+                       a["list_counts"], keys[3:], vals[3:], first_pos=n_old + 3)
+    assert np.array_equal(one["codes"], b["codes"]) and np.array_equal(one["list_ids"], b["list_ids"])
+    assert np.array_equal(one["list_counts"], b["list_counts"])
+    np.testing.assert_allclose(one["list_vmeans"], b["list_vmeans"], atol=1e-12)
+    np.testing.assert_allclose(one["key_norms"], b["key_norms"], atol=0)

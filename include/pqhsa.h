@@ -90,6 +90,18 @@ typedef struct {
                               /*                           of each list (Eq. 4); 0 if empty */
 } pqhsa_index;
 
+/* The same arrays as pqhsa_index, writable, plus the member count of every list: what
+ * pqhsa_index_update maintains.  Centroids and codebooks stay fixed (no re-clustering). */
+typedef struct {
+  const float* centroids;     /* [B][H_kv][n_list][d]                                        */
+  const float* codebooks;     /* [B][H_kv][M][256][dsub]                                     */
+  uint8_t* codes;             /* [B][H_kv][N_max][M]                                         */
+  uint16_t* list_ids;         /* [B][H_kv][N_max]                                            */
+  float* key_norms;           /* [B][H_kv][N_max]     (required here)                        */
+  float* list_vmeans;         /* [B][H_kv][n_list][d]                                        */
+  int32_t* list_counts;       /* [B][H_kv][n_list]    members behind each stored mean        */
+} pqhsa_index_rw;
+
 /* Engine-owned paged KV cache, read in place through element strides (Sec. 3.3, App. E):
  * row of (page p, slot t, KV head g) starts at  base + p*stride_page + t*stride_token +
  * g*stride_head  elements and holds d contiguous elements.  Covers both a split layout
@@ -202,6 +214,20 @@ int pqhsa_decode(const pqhsa_params* params, const void* q, const pqhsa_index* i
 int pqhsa_decode_events(const pqhsa_params* params, const void* q, const pqhsa_index* index,
                         const pqhsa_paged_kv* kv, const int32_t* seq_lens, void* out,
                         void* ws, size_t ws_bytes, void* stream, void* const* stage_events);
+
+/* Index maintenance between decode steps (Sec. 3.3, first paragraph; encoding of Sec. 3.1).
+ * For every sequence b the n_new[b] (<= max_new <= 1024) tokens at positions first_pos[b],
+ * first_pos[b] + 1, ... are read from the paged cache and encoded into the EXISTING lists:
+ * r_i = |k_i| in fp32, u_i = k_i / r_i (0 for a zero key), a_i = list of the nearest centroid
+ * to u_i (squared Euclidean distance, lower index on ties), z_im = nearest codeword to the
+ * m-th sub-vector of u_i - c_{a_i}; codes, list_ids and key_norms are written at those
+ * positions, and every list that received tokens gets vbar_j = (n_j vbar_j + sum of the new
+ * members' values) / (n_j + new_j), n_j += new_j.  first_pos / n_new: device int32 [B];
+ * positions outside [0, max_seq_len) are skipped.  Two launches on `stream`, no workspace, no
+ * synchronisation; must not overlap a decode call that reads the same index. */
+int pqhsa_index_update(const pqhsa_params* params, const pqhsa_index_rw* index,
+                       const pqhsa_paged_kv* kv, const int32_t* first_pos, const int32_t* n_new,
+                       int32_t max_new, void* stream);
 
 /* Dense decode attention over the WHOLE paged KV cache (Eq. 1 with E = every cached token):
  * softmax(q K^T / sqrt d) V per query head, split-K with a log-sum-exp merge.  Not a step of

@@ -38,6 +38,7 @@ class IvfPqIndex:
     list_ids: torch.Tensor      # [B, Hkv, N_max]            int16 storage of uint16 ids
     key_norms: torch.Tensor     # [B, Hkv, N_max]            f32
     list_vmeans: torch.Tensor   # [B, Hkv, n_list, d]        f32
+    list_counts: torch.Tensor = None   # [B, Hkv, n_list]    int32 members behind each mean
 
 
 def _assign(x: torch.Tensor, c: torch.Tensor, chunk: int = 16384):
@@ -124,7 +125,8 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
         torch.zeros((B, Hkv, Nmax, M), dtype=torch.uint8, device=dev),
         torch.zeros((B, Hkv, Nmax), dtype=torch.int16, device=dev),
         torch.zeros((B, Hkv, Nmax), dtype=torch.float32, device=dev),
-        torch.zeros((B, Hkv, nl, d), dtype=torch.float32, device=dev))
+        torch.zeros((B, Hkv, nl, d), dtype=torch.float32, device=dev),
+        torch.zeros((B, Hkv, nl), dtype=torch.int32, device=dev))
     for b in range(B):
         n = cfg.seq_lens[b]
         if n == 0:
@@ -162,4 +164,5 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
             out.list_ids[b, g, :n] = ids.to(torch.int16)
             out.key_norms[b, g, :n] = r
             out.list_vmeans[b, g] = vmean.float()
+            out.list_counts[b, g] = cnt.to(torch.int32)
     return out

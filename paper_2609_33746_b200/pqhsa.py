@@ -26,7 +26,7 @@ EXPORTS = [
     "pqhsa_decode_events", "pqhsa_decode_host", "pqhsa_last_device_status", "pqhsa_decode_buffer_offset",
     "pqhsa_decode_launch_count", "pqhsa_status_string", "pqhsa_select_static",
     "pqhsa_select_static_bytes", "pqhsa_select_static_capacity", "pqhsa_dense_decode",
-    "pqhsa_dense_workspace_bytes",
+    "pqhsa_dense_workspace_bytes", "pqhsa_index_update",
 ]
 
 
@@ -47,6 +47,11 @@ class Params(ctypes.Structure):
 class Index(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in (
         "centroids", "codebooks", "codes", "list_ids", "key_norms", "list_vmeans")]
+
+
+class IndexRW(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in (
+        "centroids", "codebooks", "codes", "list_ids", "key_norms", "list_vmeans", "list_counts")]
 
 
 class PagedKV(ctypes.Structure):
@@ -89,6 +94,7 @@ def lib() -> ctypes.CDLL:
             "pqhsa_select_static_capacity": (Z, []),
             "pqhsa_dense_decode": (I, [P, V, PK, V, V, V, Z, V]),
             "pqhsa_dense_workspace_bytes": (Z, [P]),
+            "pqhsa_index_update": (I, [P, ctypes.POINTER(IndexRW), PK, V, V, I, V]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -137,6 +143,12 @@ def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_
 def make_index(centroids, codebooks, codes, list_ids, key_norms, list_vmeans) -> Index:
     return Index(_ptr(centroids), _ptr(codebooks), _ptr(codes), _ptr(list_ids), _ptr(key_norms),
                  _ptr(list_vmeans))
+
+
+def make_index_rw(centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
+                  list_counts) -> IndexRW:
+    return IndexRW(_ptr(centroids), _ptr(codebooks), _ptr(codes), _ptr(list_ids), _ptr(key_norms),
+                   _ptr(list_vmeans), _ptr(list_counts))
 
 
 def make_paged_kv(k_cache, v_cache, stride_page, stride_token, stride_head, block_table) -> PagedKV:
@@ -256,3 +268,12 @@ def decode_host(params, q_host, q_staging, index: Index, kv: PagedKV, seq_lens, 
 
 def last_device_status(params, ws, stream=None) -> int:
     return lib().pqhsa_last_device_status(ctypes.byref(params), _ptr(ws), _stream(stream))
+
+
+def index_update(params, index_rw: IndexRW, kv: PagedKV, first_pos, n_new, max_new: int,
+                 stream=None) -> None:
+    """Encodes the tokens at positions first_pos[b] .. first_pos[b] + n_new[b] - 1 of every
+    sequence into the existing lists and refreshes the list value means (in place)."""
+    _check("pqhsa_index_update", lib().pqhsa_index_update(
+        ctypes.byref(params), ctypes.byref(index_rw), ctypes.byref(kv), _ptr(first_pos),
+        _ptr(n_new), int(max_new), _stream(stream)))

@@ -1,0 +1,164 @@
+"""Index maintenance on the GPU (pqhsa_index_update) against the oracle's index_update (-m gpu).
+
+The index of a workload is built over all its tokens; the last `n_new` tokens of every
+sequence are then taken out again (codes, ids and norms wiped, list means and counts
+recomputed over the remaining members), and the library has to put them back.  Argmin
+decisions are taken in fp32 on the GPU and in float64 by the oracle: a differing list or code
+is accepted only where the oracle's own distances say the two candidates are within fp32
+rounding of each other."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pqhsa_oracle as O
+from paper_2609_33746_b200 import pqhsa
+from paper_2609_33746_b200.runner import DecodeOp
+from paper_2609_33746_b200.workload import DecodeConfig
+
+from helpers import make_case
+
+pytestmark = pytest.mark.gpu
+
+DIST_TOL = 2e-6        # fp32 rounding of a squared distance of unit-scale vectors
+
+
+def cfg_of(name, **kw):
+    base = dict(name=name, batch=2, n_q_heads=4, n_kv_heads=2, seq_lens=(3000, 1777), dtype="bf16",
+                n_list=64, pq_m=32, budget_ppm=20000, seed=23, kmeans_iters=3)
+    base.update(kw)
+    return DecodeConfig(**base)
+
+
+CASES = {
+    "bf16_m32": (cfg_of("u1"), (256, 100)),
+    "fp16_m16_interleaved": (cfg_of("u2", dtype="fp16", pq_m=16, kv_layout="interleaved",
+                                    seq_lens=(2000, 900)), (37, 256)),
+    "m8_many_lists_one_empty_update": (cfg_of("u3", pq_m=8, n_list=256, seq_lens=(4000, 1200)),
+                                       (300, 0)),
+    "m64": (cfg_of("u4", pq_m=64, batch=1, seq_lens=(1500,)), (129,)),
+}
+
+
+@pytest.mark.parametrize("key", list(CASES))
+def test_index_update_matches_oracle(key):
+    cfg, n_new = CASES[key]
+    inp, idx = make_case(cfg, device="cuda")
+    op = DecodeOp(inp, idx)
+    B, Hkv, nl, d = cfg.batch, cfg.n_kv_heads, cfg.n_list, cfg.head_dim
+    first = [cfg.seq_lens[b] - n_new[b] for b in range(B)]
+    # take the new tokens out of the index
+    want_codes, want_ids, want_norms = idx.codes.clone(), idx.list_ids.clone(), idx.key_norms.clone()
+    vm0 = torch.zeros_like(idx.list_vmeans)
+    cnt0 = torch.zeros_like(idx.list_counts)
+    kv_rows = {}
+    for b in range(B):
+        for g in range(Hkv):
+            k, v = inp.gather_kv(b, g)
+            kv_rows[(b, g)] = (k, v)
+            ids_old = idx.list_ids[b, g, :first[b]].long() & 0xffff
+            vs = torch.zeros((nl, d), dtype=torch.float64, device="cuda").index_add_(
+                0, ids_old, v[:first[b]].double())
+            c = torch.bincount(ids_old, minlength=nl)
+            vm0[b, g] = torch.where(c[:, None] > 0, vs / c.clamp(min=1)[:, None], vs).float()
+            cnt0[b, g] = c.int()
+            idx.codes[b, g, first[b]:cfg.seq_lens[b]] = 0
+            idx.list_ids[b, g, first[b]:cfg.seq_lens[b]] = 0
+            idx.key_norms[b, g, first[b]:cfg.seq_lens[b]] = 0
+    idx.list_vmeans.copy_(vm0)
+    idx.list_counts.copy_(cnt0)
+    rw = pqhsa.make_index_rw(idx.centroids, idx.codebooks, idx.codes, idx.list_ids, idx.key_norms,
+                             idx.list_vmeans, idx.list_counts)
+    first_t = torch.tensor(first, dtype=torch.int32, device="cuda")
+    n_new_t = torch.tensor(n_new, dtype=torch.int32, device="cuda")
+    pqhsa.index_update(op.params, rw, op.kv, first_t, n_new_t, max(n_new))
+    torch.cuda.synchronize()
+
+    n_flip = 0
+    for b in range(B):
+        for g in range(Hkv):
+            k, v = kv_rows[(b, g)]
+            lo, hi = first[b], cfg.seq_lens[b]
+            ref = O.index_update(
+                idx.centroids[b, g].cpu().double().numpy(), idx.codebooks[b, g].cpu().double().numpy(),
+                want_codes[b, g].cpu().numpy() * 0, np.zeros(want_ids.shape[2], dtype=np.uint16),
+                np.zeros(want_ids.shape[2]), vm0[b, g].cpu().double().numpy(),
+                cnt0[b, g].cpu().numpy(), k[lo:hi].cpu().double().numpy(),
+                v[lo:hi].cpu().double().numpy(), first_pos=lo)
+            got_ids = (idx.list_ids[b, g, lo:hi].cpu().numpy().view(np.uint16)).astype(np.int64)
+            got_codes = idx.codes[b, g, lo:hi].cpu().numpy().astype(np.int64)
+            got_norms = idx.key_norms[b, g, lo:hi].cpu().double().numpy()
+            np.testing.assert_allclose(got_norms, ref["key_norms"][lo:hi], rtol=2e-6)
+            want_a = ref["list_ids"][lo:hi].astype(np.int64)
+            same_list = got_ids == want_a
+            for t in np.nonzero(~same_list)[0]:          # near-tie between two centroids
+                dc = ref["d_coarse"][t]
+                assert dc[got_ids[t]] - dc[want_a[t]] <= DIST_TOL, (b, g, t)
+                n_flip += 1
+            # codes are comparable where the list agrees (the residual is the same vector)
+            want_z = ref["codes"][lo:hi].astype(np.int64)
+            for t, m in zip(*np.nonzero((got_codes != want_z) & same_list[:, None])):
+                dq = ref["d_pq"][t, m]
+                assert dq[got_codes[t, m]] - dq[want_z[t, m]] <= DIST_TOL, (b, g, t, m)
+                n_flip += 1
+            # list means and counts, against the oracle run on the GPU's own assignment when
+            # it differs (a flipped token moves its value to the other list)
+            if same_list.all():
+                want_cnt, want_vm = ref["list_counts"], ref["list_vmeans"]
+            else:
+                want_cnt = cnt0[b, g].cpu().numpy().astype(np.int64) + np.bincount(got_ids, minlength=nl)
+                vs = np.zeros((nl, d))
+                np.add.at(vs, got_ids, v[lo:hi].cpu().double().numpy())
+                base = cnt0[b, g].cpu().numpy()[:, None] * vm0[b, g].cpu().double().numpy()
+                want_vm = np.where(want_cnt[:, None] > 0, (base + vs) / np.maximum(want_cnt, 1)[:, None], 0)
+            assert np.array_equal(idx.list_counts[b, g].cpu().numpy(), want_cnt)
+            np.testing.assert_allclose(idx.list_vmeans[b, g].cpu().double().numpy(), want_vm,
+                                       rtol=1e-5, atol=2e-6)
+            # nothing before the new tokens moved
+            assert torch.equal(idx.codes[b, g, :lo], want_codes[b, g, :lo])
+            assert torch.equal(idx.list_ids[b, g, :lo], want_ids[b, g, :lo])
+    total = sum(n_new) * Hkv * (1 + cfg.pq_m)
+    assert n_flip <= max(2, total // 2000), f"{n_flip} near-tie decisions of {total}"
+
+
+def test_index_update_then_decode_equals_decode_on_the_full_index():
+    """After the update the operator sees the same index as one that held the tokens from the
+    start (up to near-tie decisions, which the builder and the kernel take alike here)."""
+    cfg = cfg_of("u5", batch=1, seq_lens=(4096,), n_q_heads=4, n_kv_heads=1)
+    inp, idx = make_case(cfg, device="cuda")
+    op = DecodeOp(inp, idx)
+    op.decode()
+    torch.cuda.synchronize()
+    full = op.out.clone()
+    n_new, lo = 256, 4096 - 256
+    k, v = inp.gather_kv(0, 0)
+    ids_old = idx.list_ids[0, 0, :lo].long() & 0xffff
+    c = torch.bincount(ids_old, minlength=cfg.n_list)
+    vs = torch.zeros((cfg.n_list, 128), dtype=torch.float64, device="cuda").index_add_(0, ids_old, v[:lo].double())
+    op.list_vmeans[0, 0] = torch.where(c[:, None] > 0, vs / c.clamp(min=1)[:, None], vs).float()
+    counts = c.int().view(1, 1, -1).contiguous()
+    op.codes[0, 0, lo:] = 0
+    op.list_ids[0, 0, lo:] = 0
+    op.key_norms[0, 0, lo:] = 0
+    rw = pqhsa.make_index_rw(op.centroids, op.codebooks, op.codes, op.list_ids, op.key_norms,
+                             op.list_vmeans, counts)
+    pqhsa.index_update(op.params, rw, op.kv, torch.tensor([lo], dtype=torch.int32, device="cuda"),
+                       torch.tensor([n_new], dtype=torch.int32, device="cuda"), n_new)
+    op.decode()
+    torch.cuda.synchronize()
+    assert float((op.out.float() - full.float()).abs().max()) <= 4e-3
+
+
+def test_index_update_rejects_bad_arguments():
+    cfg = cfg_of("u6", batch=1, seq_lens=(512,), n_q_heads=2, n_kv_heads=1)
+    inp, idx = make_case(cfg, device="cuda")
+    op = DecodeOp(inp, idx)
+    rw = pqhsa.make_index_rw(op.centroids, op.codebooks, op.codes, op.list_ids, op.key_norms,
+                             op.list_vmeans, idx.list_counts)
+    z = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(pqhsa.PqhsaError) as e:
+        pqhsa.index_update(op.params, rw, op.kv, z, z, 2000)
+    assert e.value.status == pqhsa.ERR_INVALID_ARG
+    with pytest.raises(pqhsa.PqhsaError) as e:
+        pqhsa.index_update(op.params, rw, op.kv, None, z, 8)
+    assert e.value.status == pqhsa.ERR_INVALID_ARG
+    pqhsa.index_update(op.params, rw, op.kv, z, z, 0)          # nothing to do is fine

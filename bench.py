@@ -396,6 +396,8 @@ def main():
     dbytes = dense_attention_bytes(cfg, seq_lens)
     dense = dict(us_per_step=1000 * dense_ms, achieved_gbs=dbytes / (dense_ms * 1e-3) / 1e9,
                  bytes=dbytes, speedup_over_dense=dense_ms / head["ms"],
+                 ideal_us_at_measured_peak=dbytes / peak / 1e3,
+                 speedup_over_ideal_dense=(dbytes / peak / 1e6) / head["ms"],
                  kernel="dense_decode_kernel (own split-K dense decode attention, same cache)")
 
     # the same step replayed from a CUDA graph (no per-launch host work)

@@ -8,6 +8,7 @@ pqhsa_dense_decode (CUDA events, L2 flushed between steps), their ratio, and byt
 from __future__ import annotations
 
 import argparse
+import os
 import dataclasses
 import json
 import statistics
@@ -35,6 +36,17 @@ def time_call(fn, steps, flush):
     return statistics.median(a.elapsed_time(b) for a, b in ev) * 1000.0
 
 
+def copy_bandwidth_gbs():
+    """Measured device copy bandwidth if the repository carries the figure, else the pool's
+    earlier measurement."""
+    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--contexts", default="16,32,64,128,256,512", help="context lengths in K tokens")
@@ -55,10 +67,13 @@ def main():
         t_dense = time_call(lambda: pqhsa.dense_decode(op.params, op.q, op.kv, op.seq_lens, dout,
                                                        dws), args.steps, flush)
         dense_bytes = cfg.batch * cfg.n_kv_heads * cfg.max_seq_len * 2 * cfg.head_dim * 2
+        t_ideal = dense_bytes / copy_bandwidth_gbs() / 1e3      # us: one read of K and V at copy speed
         print(json.dumps(dict(context=cfg.max_seq_len, batch=cfg.batch, n_list=cfg.n_list,
                               budget_ppm=cfg.budget_ppm, pqhsa_us=round(t_pq, 1),
                               dense_us=round(t_dense, 1), dense_over_pqhsa=round(t_dense / t_pq, 3),
-                              dense_gbs=round(dense_bytes / t_dense / 1e3, 1))), flush=True)
+                              dense_gbs=round(dense_bytes / t_dense / 1e3, 1),
+                              ideal_dense_us=round(t_ideal, 1),
+                              ideal_dense_over_pqhsa=round(t_ideal / t_pq, 3))), flush=True)
         del op, inp, idx, dws
         torch.cuda.empty_cache()
 

@@ -33,6 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 512 << 20
 SCAN_DRAM_BYTES_PER_UNIT = 41.15e6 / (8 * 131072)   # ncu, profiles/scan_kernel_c3_b1.md
+SCAN_SMEM_WAVEFRONTS_PER_TILE = 176      # l1tex__data_pipe_lsu_wavefronts_mem_shared / tiles, same capture
 
 
 def measured_peak():
@@ -336,6 +337,12 @@ def main():
                     stage_ms=dict(lut=stage_ms[0], scan=stage_ms[1], select=stage_ms[2],
                                   attend=stage_ms[3]),
                     whole_step_frac_of_peak=head["gbs"] / world / peak)
+    # the unit that binds the scan: one shared-memory wavefront per SM and clock.  ncu counted
+    # 176 wavefronts per 32-token tile of a (KV head, 4-head group) on c3_b1
+    # (profiles/scan_kernel_c3_b1.md); the clock is the median sampled below, filled in later.
+    scan_tiles = cfg.n_kv_heads * ((cfg.group + 3) // 4) * sum((n + 31) // 32 for n in seq_lens)
+    roofline["shared_memory_pipe"] = dict(wavefronts_per_tile=SCAN_SMEM_WAVEFRONTS_PER_TILE,
+                                          tiles_per_launch=scan_tiles)
 
     # end to end through the host-buffer entry point: q from pinned host memory, out back
     q_host = op.q.cpu().pin_memory()
@@ -450,6 +457,15 @@ def main():
         del codes2, ids2, norms2, vm2, cnt2
 
     clocks = sampler.stop()              # sampled over every timed loop above
+    try:      # an auxiliary figure: never let it cost the JSON line
+        if clocks.get("sm_mhz"):
+            sp = roofline["shared_memory_pipe"]
+            n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+            cycles = stage_ms[1] * 1e-3 * clocks["sm_mhz"] * 1e6
+            sp["frac_of_one_wavefront_per_sm_clock"] = (
+                sp["wavefronts_per_tile"] * sp["tiles_per_launch"] / n_sm / cycles)
+    except Exception:
+        pass
     cpu_baseline = None
     if rank == 0 and world == 1:
         # whole sequences (all query heads), one after the other, until about 10 s of oracle time

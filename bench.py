@@ -10,6 +10,15 @@ resident in HBM.  Prints ONE JSON line (rank 0).
 Under torchrun (N > 1) every rank runs the same workload on its own GPU with its own seed
 (the operator shards over sequences with no exchange step): weak scaling, value = the sum
 over ranks of algorithmic bytes / max-over-ranks step time.
+
+Beside the contract keys the line carries: `roofline` (the scan kernel against the measured
+copy bandwidth, its DRAM traffic from an ncu capture, per-stage times from
+pqhsa_decode_events and the utilisation of the shared-memory pipe, which is what binds the
+scan), `e2e` (pqhsa_decode_host: query from pinned host memory, output read back),
+`cpu_baseline` (the float64 oracle on whole sequences for about 10 s), `variants` (the other
+config-3 shapes), `dense_comparator` (the library's dense decode kernel on the same cache,
+and the ideal time of one read of K and V), `graph_replay_us_per_step` and `index_update`
+(index maintenance, amortised over the 256 steps between two calls).
 """
 from __future__ import annotations
 
@@ -47,7 +56,7 @@ def measured_peak():
 
 # ------------------------------------------------------------------ algorithmic bytes
 def algorithmic_bytes(cfg, seq_lens, budget_ppm):
-    """Bytes one step must move ("Algorithmic bytes").  Per sequence and KV head:
+    """Bytes one step must move.  Per sequence and KV head:
     codes M + norm 4 + list id 2 per token; one score row per query head written once and
     read once (4+4 B per token per query head); k exact K and V rows of 2*d*2 B per query
     head plus 64 B for the two 32-byte sectors that return the token's score and list id;

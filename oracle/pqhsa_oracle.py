@@ -21,7 +21,7 @@ re-ordering:
     O10 index maintenance: new tokens encoded into the existing lists,  (Sec. 3.3, first paragraph;
         list means refreshed, no re-clustering                           Sec. 3.1 for the encoding)
 
-Readings where the paper is silent (each also listed in the design doc):
+Readings where the paper is silent (the repository's design notes list them too):
   * top-k ties: stable, the lower position wins;
   * rho is given in parts per million and k is computed in integers;
   * u_q = 0 when r_q = 0;

@@ -27,12 +27,23 @@ CASES = [
     ("c3_b8_r1", [(0, 3), (4, 20), (7, 31)]),          # the benchmark's default workload
     ("c4", [(2, 7), (11, 30)]),                        # ragged batch of 16, G = 8
     ("c5_n512_b1", [(0, 1), (0, 30)]),                 # 512K context, n_list = 4096
+    # the paper's own partition at 128K: 4 sinks, 128-token window, exact set in whole pages
+    # (1,456 tokens at 1 %, App. A)
+    ("c3_b1_r1+sinks_window_pages", [(0, 2), (0, 27)]),
 ]
+
+
+def config_of(name):
+    base, _, extra = name.partition("+")
+    cfg = named_config(base)
+    if extra == "sinks_window_pages":
+        cfg = dataclasses.replace(cfg, n_sink=4, n_local=128, exact_set_multiple=16)
+    return cfg
 
 
 @pytest.mark.parametrize("name,rows", CASES, ids=[c[0] for c in CASES])
 def test_full_size_decode_on_sampled_rows(name, rows):
-    cfg = dataclasses.replace(named_config(name), kmeans_iters=2)
+    cfg = dataclasses.replace(config_of(name), kmeans_iters=2)
     inp = generate(cfg, device="cuda")
     idx = build_index(inp)
     op = DecodeOp(inp, idx)
@@ -51,13 +62,16 @@ def test_full_size_decode_on_sampled_rows(name, rows):
         sub = dataclasses.replace(inp, cfg=dataclasses.replace(cfg, batch=1, seq_lens=(cfg.seq_lens[b],)))
         ref = run_oracle(sub, None, heads=heads, batch_items=[0], arrays=arrays)
         n = cfg.seq_lens[b]
+        r0, r1 = min(cfg.n_sink, n), max(min(cfg.n_sink, n), n - cfg.n_local)     # R = [r0, r1)
         for h in heads:
             r = ref[(0, h)]
-            got = scores[b, h, :n].cpu().double().numpy()
+            got = scores[b, h, r0:r1].cpu().double().numpy()
             assert np.all(np.abs(got - r["approx"]) <= LOGIT_RTOL * np.maximum(np.abs(r["approx"]), 1.0)), \
                 f"{name} logits row {(b, h)}: {np.abs(got - r['approx']).max()}"
             c = int(cnt[b, h])
             assert c == r["k"]
+            if cfg.exact_set_multiple > 1:
+                assert (c + r0 + (n - r1)) % cfg.exact_set_multiple == 0
             ok, why = selection_matches(sel[b, h, :c].cpu().numpy(), r)
             assert ok, f"{name} selection row {(b, h)}: {why}"
             y = out[b, h].cpu().double().numpy()

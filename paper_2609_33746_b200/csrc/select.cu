@@ -21,7 +21,8 @@ namespace pqhsa {
 namespace {
 
 constexpr int kElems = kSelChunk / kSelThreads;   // scores per thread per chunk (16)
-constexpr int kStashCap = 3072;                   // candidates resolved from shared memory
+constexpr int kStashCap = 5120;                   // candidates resolved from shared memory
+constexpr int kFilterSmemBytes = kHistBins * 4 + kStashCap * 8;   // dynamic: above the 48 KB static limit
 constexpr int kSample = 4096;                     // sampled scores per row
 constexpr int kSamplePer = kSample / kSelThreads; // per thread (8)
 constexpr int kSampleGroups = kSample / 4;        // groups of 4 consecutive scores
@@ -361,7 +362,7 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
                   float* __restrict__ kth, int* __restrict__ status) {
   // main pass: a 512-entry hit buffer per warp; last CTA: histogram + candidate stash.
   // The two uses never overlap in time, so they share the same shared memory.
-  __shared__ __align__(16) unsigned char s_raw[kHistBins * 4 + kStashCap * 8];
+  extern __shared__ __align__(16) unsigned char s_raw[];          // kFilterSmemBytes
   uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_raw);
   uint2* s_stash = reinterpret_cast<uint2*>(s_raw + kHistBins * 4);
   uint32_t* s_hits = reinterpret_cast<uint32_t*>(s_raw);          // [16 warps][512]
@@ -476,7 +477,7 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
     } else {
       int src = kFromList;
       if (C <= kStashCap) {
-        constexpr int kPer = kStashCap / kSelThreads;          // 6: all loads issued together
+        constexpr int kPer = kStashCap / kSelThreads;          // 10: all loads issued together
         int pos[kPer];
         float sc[kPer];
 #pragma unroll
@@ -522,7 +523,12 @@ cudaError_t launch_select(const Plan& pl, const WsLayout& L, char* ws, const flo
   cudaError_t e = launch_pdl(sel_sample_kernel, dim3(pl.rows), dim3(kSelThreads), 0, st, pl, scores,
                              seq_lens, rowstate, sel_count, kth);
   if (e != cudaSuccess) return e;
-  return launch_pdl(sel_filter_kernel, dim3(pl.hist_chunks, pl.rows), dim3(kSelThreads), 0, st, pl,
+  // more than 48 KB of dynamic shared memory needs an opt-in (per device, so set every time)
+  e = cudaFuncSetAttribute(sel_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kFilterSmemBytes);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(sel_filter_kernel, dim3(pl.hist_chunks, pl.rows), dim3(kSelThreads),
+                    kFilterSmemBytes, st, pl,
                     scores, counters, rowstate, cand, sel_idx, sel_count, kth, status);
 }
 

@@ -115,6 +115,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   // background preparation: CTAs per row
   o.bg_ctas = ceil_div(2LL * o.num_sms, o.rows);
   if (o.bg_ctas > 8) o.bg_ctas = 8;
+  if (o.bg_ctas < ceil_div(o.k_max, 768)) o.bg_ctas = ceil_div(o.k_max, 768);   // 6 tokens per thread
   if (o.bg_ctas < 1) o.bg_ctas = 1;
 #ifdef PQHSA_TUNE
   if (const char* e = getenv("PQHSA_HIST_CHUNKS")) o.hist_chunks = atoi(e);

@@ -17,7 +17,7 @@ namespace pqhsa {
 
 namespace {
 
-constexpr int kBgThreads = 256;
+constexpr int kBgThreads = 128;
 constexpr int kMaxSeg = 160;                  // >= n_part for any plan (148 SMs / 1 unit + 2)
 
 // grid (bg_ctas, rows).  CTA c merges a slice of the lists and subtracts a slice of the
@@ -48,7 +48,7 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
   const float* rs = scores + (size_t)row * pl.N_max;
   const uint16_t* rl = lids + ((size_t)b * pl.Hkv + kv) * pl.N_max;
-  constexpr int kSelPer = 4;
+  constexpr int kSelPer = 6;
   int idx[kSelPer];
   float sc[kSelPer];
   uint32_t li[kSelPer];

@@ -384,11 +384,53 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
   uint32_t* n_cand = &counters[row * 4 + 3];
 
   // Main pass.  Warps work independently: a lane marks which of its 16 scores reach the
-  // bracket, the warp packs the positions of the hits (bit 31 = certain winner) into its
-  // shared-memory buffer, and flushes them with one atomic per destination list.
+  // bracket and the warp packs the positions of the hits (bit 31 = certain winner) into its
+  // shared-memory buffer.  The buffer is written out when it would overflow and at the end,
+  // with one atomic per destination list, so the round trip of that atomic is paid once per
+  // warp and not once per chunk.
   const int n_chunks = (n + kSelChunk - 1) / kSelChunk;
   const bool no_winners = !(hi_f < CUDART_INF_F);   // bracket open at the top: candidates only
-  uint32_t* my_hits = s_hits + warp * (kSelChunk / 16);
+  constexpr int kBuf = kSelChunk / 16;              // entries per warp: one chunk's worst case
+  uint32_t* my_hits = s_hits + warp * kBuf;
+  int buf_n = 0;                                    // warp-uniform
+  auto flush = [&]() {
+    if (buf_n == 0) return;
+    int nw = 0, nc = 0;
+    for (int i0 = 0; i0 < buf_n; i0 += 32) {
+      const bool v_ok = i0 + lane < buf_n;
+      const uint32_t ent = v_ok ? my_hits[i0 + lane] : 0u;
+      nw += __popc(__ballot_sync(0xffffffffu, v_ok && (ent >> 31)));
+      nc += __popc(__ballot_sync(0xffffffffu, v_ok && !(ent >> 31)));
+    }
+    uint32_t bw = 0, bc = 0;
+    if (lane == 0) {
+      if (nw) bw = atomicAdd(n_out, (uint32_t)nw);
+      if (nc) bc = atomicAdd(n_cand, (uint32_t)nc);
+    }
+    bw = __shfl_sync(0xffffffffu, bw, 0);
+    bc = __shfl_sync(0xffffffffu, bc, 0);
+    const unsigned lt = (1u << lane) - 1u;
+    for (int i0 = 0; i0 < buf_n; i0 += 32) {
+      const bool v_ok = i0 + lane < buf_n;
+      const uint32_t ent = v_ok ? my_hits[i0 + lane] : 0u;
+      const bool is_win = v_ok && (ent >> 31);
+      const bool is_cnd = v_ok && !(ent >> 31);
+      const unsigned mw = __ballot_sync(0xffffffffu, is_win);
+      const unsigned mc = __ballot_sync(0xffffffffu, is_cnd);
+      if (is_win) {
+        const uint32_t p = bw + __popc(mw & lt);
+        if (p < (uint32_t)pl.k_max) out[p] = (int)(ent & 0x7fffffffu);
+      }
+      if (is_cnd) {
+        const uint32_t p = bc + __popc(mc & lt);
+        if (p < (uint32_t)pl.cand_cap) rc[p] = (int)ent;
+      }
+      bw += __popc(mw);
+      bc += __popc(mc);
+    }
+    __syncwarp();
+    buf_n = 0;
+  };
   for (int ch = chunk; ch < n_chunks; ch += gridDim.x) {
     float v[kElems];
     int pos0[4];
@@ -416,7 +458,8 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
     }
     const int total = __shfl_sync(0xffffffffu, inc, 31);
     if (total == 0) continue;                        // warp-uniform
-    int slot = inc - mine;
+    if (buf_n + total > kBuf) flush();
+    int slot = buf_n + inc - mine;
     const int pos_base = ch * kSelChunk + tid * 4;   // position of element e: + (e>>2)*2048 + (e&3)
     while (hit) {
       const int e = __ffs(hit) - 1;
@@ -425,33 +468,9 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
                         (((win >> e) & 1u) << 31);
     }
     __syncwarp();
-    for (int i0 = 0; i0 < total; i0 += 32) {
-      const int i = i0 + lane;
-      const bool v_ok = i < total;
-      const uint32_t ent = v_ok ? my_hits[i] : 0u;
-      const bool is_win = v_ok && (ent >> 31);
-      const bool is_cnd = v_ok && !(ent >> 31);
-      const unsigned mw = __ballot_sync(0xffffffffu, is_win);
-      const unsigned mc = __ballot_sync(0xffffffffu, is_cnd);
-      uint32_t bw = 0, bc = 0;
-      if (lane == 0) {
-        if (mw) bw = atomicAdd(n_out, (uint32_t)__popc(mw));
-        if (mc) bc = atomicAdd(n_cand, (uint32_t)__popc(mc));
-      }
-      bw = __shfl_sync(0xffffffffu, bw, 0);
-      bc = __shfl_sync(0xffffffffu, bc, 0);
-      const unsigned lt = (1u << lane) - 1u;
-      if (is_win) {
-        const uint32_t p = bw + __popc(mw & lt);
-        if (p < (uint32_t)pl.k_max) out[p] = (int)(ent & 0x7fffffffu);
-      }
-      if (is_cnd) {
-        const uint32_t p = bc + __popc(mc & lt);
-        if (p < (uint32_t)pl.cand_cap) rc[p] = (int)ent;
-      }
-    }
-    __syncwarp();
+    buf_n += total;
   }
+  flush();
   if (!cta_arrived_last(&counters[row * 4 + 1], gridDim.x, &s_last)) return;
 
   // ---- last CTA of the row: check the bracket by counting, then select among the candidates

@@ -68,6 +68,16 @@ CASES = {
                                        n_q_heads=4, n_kv_heads=1, n_sink=4, n_local=128,
                                        exact_set_multiple=16),
     "window_only_g8": small("w8", n_q_heads=16, n_kv_heads=2, seq_lens=(2500,), n_local=64),
+    # other page sizes of the engine's cache, down to one token per page
+    "pages_of_32": small("p32", page_size=32, seq_lens=(3100,), n_q_heads=4, n_kv_heads=1),
+    "pages_of_1": small("p1", page_size=1, seq_lens=(1008,), n_q_heads=4, n_kv_heads=2),
+    # the widest GQA group the library takes: 16 query heads on one KV head, 4 head groups
+    "g16_four_head_groups": small("g16", n_q_heads=16, n_kv_heads=1, seq_lens=(2300,)),
+    # a budget of one token per row
+    "budget_of_one_token": small("k1", seq_lens=(5000,), budget_ppm=100, n_q_heads=4, n_kv_heads=1),
+    # the largest list count, most lists empty
+    "lists_4096_mostly_empty": small("l4096", seq_lens=(3000,), n_list=4096, n_q_heads=4,
+                                     n_kv_heads=1, kmeans_iters=1),
 }
 
 

@@ -25,7 +25,8 @@
  *   - Arguments are validated on the host first; on error nothing is launched and a
  *     negative pqhsa_status is returned.  PQHSA_OK (0) means "launched", not "finished".
  *   - Input arrays are read-only.  Rows past seq_lens[b] are never read.
- *   - v1 limits: head_dim == 128; pq_ncode == 256 (uint8 codes); pq_m in {8,16,32,64} with
+ *   - v1 limits: head_dim == 128; pq_ncode == 256 (one byte per code, pq_m in {8,16,32,64}) or
+ *     pq_ncode == 16 (two 4-bit codes per byte, pq_m in {8,16}: the paper's own index setting) with
  *     pq_m * pq_dsub == 128; n_list <= 4096 (and the per-CTA tables must fit shared memory,
  *     see PQHSA_ERR_UNSUPPORTED); max_seq_len % 4 == 0; page rows 16-byte aligned
  *     (strides multiples of 8 elements).
@@ -60,7 +61,7 @@ typedef struct {
   int32_t n_list;             /* inverted lists per (sequence, KV head)                     */
   int32_t pq_m;               /* M  PQ subspaces                                            */
   int32_t pq_dsub;            /* dims per subspace, M * dsub == d                           */
-  int32_t pq_ncode;           /* 2^b codewords per subspace (256)                           */
+  int32_t pq_ncode;           /* 2^b codewords per subspace: 256 or 16                       */
   int32_t max_seq_len;        /* N_max: row stride of codes / list_ids / key_norms / scores */
   int32_t page_size;          /* tokens per KV page                                         */
   int32_t max_pages_per_seq;  /* row stride of block_table                                  */
@@ -83,7 +84,8 @@ typedef struct {
   const float* centroids;     /* [B][H_kv][n_list][d]      c_j                              */
   const float* codebooks;     /* [B][H_kv][M][256][dsub]   p_{m,z}; subspace m = dims       */
                               /*                           [m*dsub, (m+1)*dsub)             */
-  const uint8_t* codes;       /* [B][H_kv][N_max][M]       z_im                             */
+  const uint8_t* codes;       /* [B][H_kv][N_max][M]       z_im; with pq_ncode == 16         */
+                              /* [B][H_kv][N_max][M/2]: byte j = z_{i,2j} | z_{i,2j+1} << 4   */
   const uint16_t* list_ids;   /* [B][H_kv][N_max]          a_i < n_list                     */
   const float* key_norms;     /* [B][H_kv][N_max]          r_i, or NULL for all ones        */
   const float* list_vmeans;   /* [B][H_kv][n_list][d]      stored mean value of ALL members */

@@ -56,8 +56,14 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (k_need > p->max_seq_len) k_need = p->max_seq_len;
   if (p->k_max < k_need) return PQHSA_ERR_INVALID_ARG;
 
-  if (p->head_dim != kHeadDim || p->pq_ncode != kNCode) return PQHSA_ERR_UNSUPPORTED;
-  if (p->pq_m != 8 && p->pq_m != 16 && p->pq_m != 32 && p->pq_m != 64) return PQHSA_ERR_UNSUPPORTED;
+  if (p->head_dim != kHeadDim) return PQHSA_ERR_UNSUPPORTED;
+  if (p->pq_ncode == 256) {
+    if (p->pq_m != 8 && p->pq_m != 16 && p->pq_m != 32 && p->pq_m != 64) return PQHSA_ERR_UNSUPPORTED;
+  } else if (p->pq_ncode == 16) {      // 4-bit codes, two per byte (the paper's own index setting)
+    if (p->pq_m != 8 && p->pq_m != 16) return PQHSA_ERR_UNSUPPORTED;
+  } else {
+    return PQHSA_ERR_UNSUPPORTED;
+  }
   if (p->n_list > 4096 || p->max_seq_len % 4 != 0) return PQHSA_ERR_UNSUPPORTED;
   const int G = p->n_q_heads / p->n_kv_heads;
   if (G > 16) return PQHSA_ERR_UNSUPPORTED;
@@ -67,6 +73,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.Gc = G <= 2 ? G : 4;
   o.n_hg = (G + o.Gc - 1) / o.Gc;
   o.n_list = p->n_list; o.M = p->pq_m; o.dsub = p->pq_dsub;
+  o.n_code = p->pq_ncode; o.code_bytes = p->pq_ncode == 16 ? p->pq_m / 2 : p->pq_m;
   o.N_max = p->max_seq_len; o.page_size = p->page_size; o.max_pages = p->max_pages_per_seq;
   o.k_max = p->k_max; o.n_sink = p->n_sink; o.n_local = p->n_local;
   o.exact_multiple = p->exact_set_multiple; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
@@ -129,7 +136,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
 static size_t buffer_elems(const Plan& pl, int which) {
   const size_t units = (size_t)pl.B * pl.Hkv * pl.n_hg;
   switch (which) {
-    case PQHSA_BUF_LUT: return units * kNCode * pl.M * pl.Gc;
+    case PQHSA_BUF_LUT: return units * pl.n_code * pl.M * pl.Gc;
     case PQHSA_BUF_COARSE: return units * pl.n_list * pl.Gc;
     case PQHSA_BUF_SCORES: return (size_t)pl.rows * pl.N_max;
     case PQHSA_BUF_LIST_PARTIALS: return (size_t)pl.rows * pl.n_part * (pl.n_list + 1);

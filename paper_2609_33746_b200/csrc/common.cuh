@@ -30,6 +30,8 @@ constexpr float kNegligibleLog2 = -40.0f;   // exp2 arguments below this are lef
 struct Plan {
   int B, Hq, Hkv, G, Gc, n_hg;       // Gc heads per scan pass, n_hg = ceil(G / Gc)
   int n_list, M, dsub;
+  int n_code;                        // codewords per subspace: 256 (one byte per code) or 16 (two codes per byte)
+  int code_bytes;                    // bytes of codes per token: M or M / 2
   int N_max, page_size, max_pages;
   int k_max;
   int n_sink, n_local;               // |S| and |L| of Sec. 3.2 (upper bounds: clipped per sequence)

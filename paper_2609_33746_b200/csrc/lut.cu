@@ -70,7 +70,7 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
   const int rows_per_cta = (pl.n_list + kLutChunks - 1) / kLutChunks;
   const int r0 = blockIdx.x * rows_per_cta;
   const int r1 = min(pl.n_list, r0 + rows_per_cta);
-  constexpr int kEntPerM = kNCode;
+  const int kEntPerM = pl.n_code;
   const int n_ent = pl.M * kEntPerM;
   const int ent_per_cta = (n_ent + kLutChunks - 1) / kLutChunks;
   const int e0 = blockIdx.x * ent_per_cta;
@@ -165,7 +165,7 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
           for (int t = 0; t < DSUB; ++t) v[g] = fmaf(cw[t], qs[t], v[g]);
         }
       }
-      float* dst = lut + (((ukv * n_hg + hg) * kNCode + z) * pl.M + m) * Gc;
+      float* dst = lut + (((ukv * n_hg + hg) * pl.n_code + z) * pl.M + m) * Gc;
       if (Gc == 4) *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
       else if (Gc == 2) *reinterpret_cast<float2*>(dst) = make_float2(v[0], v[1]);
       else dst[0] = v[0];

@@ -97,7 +97,7 @@ __device__ __forceinline__ void load_meta(TokenMeta& r, const uint16_t* __restri
   }
 }
 
-// ---- per-warp cp.async ring for the code tiles
+// ---- per-warp cp.async ring for the code tiles; M here = bytes of codes per token
 template <int M> struct CodeTile {
   static constexpr int kChunkBytes = M < 16 ? M : 16;       // one cp.async
   static constexpr int kChunksPerToken = M / kChunkBytes;   // C
@@ -110,11 +110,13 @@ template <int M> struct CodeTile {
   }
 };
 
-__device__ __forceinline__ void cp_async(uint32_t dst, const void* src, int bytes16) {
-  if (bytes16)
+template <int kBytes> __device__ __forceinline__ void cp_async(uint32_t dst, const void* src) {
+  if constexpr (kBytes == 16)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-  else
+  else if constexpr (kBytes == 8)
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+  else
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() {
   asm volatile("cp.async.commit_group;" ::: "memory");
@@ -135,8 +137,8 @@ __device__ __forceinline__ void issue_tile(uint32_t slot, const uint8_t* __restr
       const int tok = q / CT::kChunksPerToken, c = q % CT::kChunksPerToken;
       const int i = t * kTile + tok;
       if (i < Nb)
-        cp_async(slot + tok * M + ((c ^ CT::swz(tok)) * CT::kChunkBytes),
-                 codes + (row_base + i) * M + c * CT::kChunkBytes, CT::kChunkBytes == 16);
+        cp_async<CT::kChunkBytes>(slot + tok * M + ((c ^ CT::swz(tok)) * CT::kChunkBytes),
+                                  codes + (row_base + i) * M + c * CT::kChunkBytes);
     }
   }
   cp_async_commit();
@@ -147,7 +149,9 @@ template <int M>
 __device__ __forceinline__ void read_codes(uint32_t slot, int lane, uint32_t (&w)[M / 4]) {
   using CT = CodeTile<M>;
   const uint32_t tok_addr = slot + lane * M;
-  if constexpr (M == 8) {
+  if constexpr (M == 4) {
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(w[0]) : "r"(tok_addr));
+  } else if constexpr (M == 8) {
     asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "r"(tok_addr));
   } else {
 #pragma unroll
@@ -189,13 +193,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return false;
 }
 
-template <int M, int GC, int kStages>
+// kBits = 8: one byte per code, 256-entry tables.  kBits = 4: two codes per byte (subspace 2j in
+// the low nibble of byte j), 16-entry tables.
+template <int M, int GC, int kStages, int kBits>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restrict__ lids,
             const float* __restrict__ norms, const float* __restrict__ lut,
             const float* __restrict__ coarse, const int32_t* __restrict__ seq_lens,
             float* __restrict__ scores, float* __restrict__ partials, int* __restrict__ status) {
-  constexpr int kLutFloats = kNCode * M * GC;
+  constexpr int kCodes = kBits == 4 ? 16 : 256;       // codewords per subspace
+  constexpr int kCB = kBits == 4 ? M / 2 : M;         // bytes of codes per token
+  constexpr int kLutFloats = kCodes * M * GC;
   constexpr int kEntryBytes = GC * 4;
   constexpr int kRowBytes = M * kEntryBytes;       // stride between consecutive z
   constexpr int kWarps = kScanThreads / 32;
@@ -212,7 +220,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   const uint32_t table_bytes =
       uint32_t(kLutFloats + GC * pl.n_list * (pl.coarse_in_smem ? 2 : 1)) * 4u;
   const uint32_t ring0 = smem_u32(smem_raw) + ((table_bytes + 127u) & ~127u) +
-                         uint32_t((threadIdx.x >> 5) * kStages * CodeTile<M>::kBytes);
+                         uint32_t((threadIdx.x >> 5) * kStages * CodeTile<kCB>::kBytes);
   __shared__ float s_red[kWarps][GC];
   __shared__ float s_ref[GC], s_max[GC];
   __shared__ int s_overflow;
@@ -289,8 +297,8 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     int t = t0 + warp;
 #pragma unroll
     for (int st = 0; st < kStages - 1; ++st)
-      issue_tile<M>(ring0 + st * CodeTile<M>::kBytes, codes, row_base, t + st * kWarps, tend, Nb,
-                    lane);
+      issue_tile<kCB>(ring0 + st * CodeTile<kCB>::kBytes, codes, row_base, t + st * kWarps, tend,
+                      Nb, lane);
     TokenMeta cur;
     load_meta(cur, lids, norms, row_base, t * kTile + lane, t < tend && t * kTile + lane < Nb);
     if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, 4);
@@ -307,7 +315,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
       const bool have = t < tend;
       const int tn = t + kWarps;
       __syncwarp();      // every lane is done reading the slot that is refilled next
-      issue_tile<M>(ring0 + ((it + kStages - 1) % kStages) * CodeTile<M>::kBytes, codes, row_base,
+      issue_tile<kCB>(ring0 + ((it + kStages - 1) % kStages) * CodeTile<kCB>::kBytes, codes, row_base,
                     t + (kStages - 1) * kWarps, tend, Nb, lane);
       TokenMeta nxt;
       load_meta(nxt, lids, norms, row_base, tn * kTile + lane, tn < tend && tn * kTile + lane < Nb);
@@ -321,6 +329,30 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
       for (int g = 0; g < GC; ++g) sc[g] = -CUDART_INF_F;
 
       if (have) {
+        Acc<GC> acc0, acc1;
+        acc0.zero();
+        acc1.zero();
+        if constexpr (kBits == 4) {
+          // nibble m of the lane's code word(s); at step s the lane looks up m = s ^ (lane & 7)
+          // inside its group of 8 subspaces, as in the 8-bit path
+          uint32_t cw4[kCB / 4];
+          read_codes<kCB>(ring0 + (it % kStages) * CodeTile<kCB>::kBytes, lane, cw4);
+#pragma unroll
+          for (int sb = 0; sb < M; sb += kBlk) {
+            Acc<GC> v[kBlk];
+#pragma unroll
+            for (int u = 0; u < kBlk; ++u) {
+              const int s = sb + u;
+              const uint32_t z = (cw4[s >> 3] >> (4 * ((s & 7) ^ lx))) & 15u;
+              v[u].load(lane_off[s & 7] + z * uint32_t(kRowBytes) + uint32_t((s & ~7) * kEntryBytes));
+            }
+#pragma unroll
+            for (int u = 0; u < kBlk; u += 2) {
+              acc0.merge(v[u]);
+              acc1.merge(v[u + 1]);
+            }
+          }
+        } else {
         // position p of the lane's code array <- original byte p ^ (lane & 7)
         uint32_t raw[M / 4], cw[M / 4];
         read_codes<M>(ring0 + (it % kStages) * CodeTile<M>::kBytes, lane, raw);
@@ -330,9 +362,6 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
           cw[2 * j] = __byte_perm(swap_words ? bb : a, 0u, byte_sel);
           cw[2 * j + 1] = __byte_perm(swap_words ? a : bb, 0u, byte_sel);
         }
-        Acc<GC> acc0, acc1;
-        acc0.zero();
-        acc1.zero();
 #pragma unroll
         for (int sb = 0; sb < M; sb += kBlk) {
           Acc<GC> v[kBlk];
@@ -347,6 +376,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
             acc0.merge(v[u]);
             acc1.merge(v[u + 1]);
           }
+        }
         }
         acc0.merge(acc1);
         float accf[GC], co[GC];
@@ -465,21 +495,21 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
 }
 
 size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem, int stages) {
-  size_t f = (size_t)kNCode * pl.M * pl.Gc + (size_t)pl.Gc * pl.n_list;
+  size_t f = (size_t)pl.n_code * pl.M * pl.Gc + (size_t)pl.Gc * pl.n_list;
   if (coarse_in_smem) f += (size_t)pl.Gc * pl.n_list;
   const size_t tables = (f * sizeof(float) + 127) / 128 * 128;    // the ring is 128-byte aligned
-  return tables + (size_t)(kScanThreads / 32) * stages * kTile * pl.M;
+  return tables + (size_t)(kScanThreads / 32) * stages * kTile * pl.code_bytes;
 }
 
-template <int M, int GC, int S>
+template <int M, int GC, int S, int kBits>
 static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const float* lut,
                                  const float* coarse, const int32_t* seq_lens, float* scores,
                                  float* partials, int* status, cudaStream_t st) {
   const size_t smem = scan_smem_bytes(pl, pl.coarse_in_smem != 0, S);
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S>,
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S, kBits>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(scan_kernel<M, GC, S>, dim3(pl.scan_ctas), dim3(kScanThreads), smem, st, pl,
+  return launch_pdl(scan_kernel<M, GC, S, kBits>, dim3(pl.scan_ctas), dim3(kScanThreads), smem, st, pl,
                     ix.codes, ix.list_ids, ix.key_norms, lut, coarse, seq_lens, scores, partials,
                     status);
 }
@@ -487,18 +517,20 @@ static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const fl
 cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,
                         const float* coarse, const int32_t* seq_lens, float* scores,
                         float* list_partials, int* status, cudaStream_t st) {
-#define PQHSA_SCAN_CASE(MM, GG)                                                               \
-  if (pl.M == MM && pl.Gc == GG) {                                                            \
+#define PQHSA_SCAN_CASE(MM, GG, BITS)                                                         \
+  if (pl.M == MM && pl.Gc == GG && pl.n_code == (BITS == 4 ? 16 : 256)) {                     \
     if (pl.scan_stages >= 3)                                                                  \
-      return launch_scan_t<MM, GG, 3>(pl, ix, lut, coarse, seq_lens, scores, list_partials,   \
-                                      status, st);                                            \
-    return launch_scan_t<MM, GG, 2>(pl, ix, lut, coarse, seq_lens, scores, list_partials,     \
-                                    status, st);                                              \
+      return launch_scan_t<MM, GG, 3, BITS>(pl, ix, lut, coarse, seq_lens, scores,            \
+                                            list_partials, status, st);                       \
+    return launch_scan_t<MM, GG, 2, BITS>(pl, ix, lut, coarse, seq_lens, scores,              \
+                                          list_partials, status, st);                         \
   }
-  PQHSA_SCAN_CASE(8, 1) PQHSA_SCAN_CASE(8, 2) PQHSA_SCAN_CASE(8, 4)
-  PQHSA_SCAN_CASE(16, 1) PQHSA_SCAN_CASE(16, 2) PQHSA_SCAN_CASE(16, 4)
-  PQHSA_SCAN_CASE(32, 1) PQHSA_SCAN_CASE(32, 2) PQHSA_SCAN_CASE(32, 4)
-  PQHSA_SCAN_CASE(64, 1) PQHSA_SCAN_CASE(64, 2)
+  PQHSA_SCAN_CASE(8, 1, 8) PQHSA_SCAN_CASE(8, 2, 8) PQHSA_SCAN_CASE(8, 4, 8)
+  PQHSA_SCAN_CASE(16, 1, 8) PQHSA_SCAN_CASE(16, 2, 8) PQHSA_SCAN_CASE(16, 4, 8)
+  PQHSA_SCAN_CASE(32, 1, 8) PQHSA_SCAN_CASE(32, 2, 8) PQHSA_SCAN_CASE(32, 4, 8)
+  PQHSA_SCAN_CASE(64, 1, 8) PQHSA_SCAN_CASE(64, 2, 8)
+  PQHSA_SCAN_CASE(8, 1, 4) PQHSA_SCAN_CASE(8, 2, 4) PQHSA_SCAN_CASE(8, 4, 4)
+  PQHSA_SCAN_CASE(16, 1, 4) PQHSA_SCAN_CASE(16, 2, 4) PQHSA_SCAN_CASE(16, 4, 4)
 #undef PQHSA_SCAN_CASE
   return cudaErrorInvalidValue;
 }

@@ -124,9 +124,9 @@ index_encode_kernel(Plan pl, const T* __restrict__ kc, long long stride_page, lo
     int bz[kUpdTok];
 #pragma unroll
     for (int t = 0; t < kUpdTok; ++t) { bd[t] = CUDART_INF_F; bz[t] = 0; }
-    const float* cb = codebooks + (ukv * pl.M + m) * (size_t)kNCode * DSUB;
-    for (int i = 0; i < kNCode / 32; ++i) {
-      const int z = lane + 32 * i;
+    const float* cb = codebooks + (ukv * pl.M + m) * (size_t)pl.n_code * DSUB;
+    for (int z0 = 0; z0 < pl.n_code; z0 += 32) {
+      const int z = min(z0 + lane, pl.n_code - 1);      // lanes past the codebook repeat its last word
       float p[DSUB];
       if constexpr (DSUB == 2) {
         const float2 v = __ldg(reinterpret_cast<const float2*>(cb + (size_t)z * DSUB));
@@ -161,10 +161,13 @@ index_encode_kernel(Plan pl, const T* __restrict__ kc, long long stride_page, lo
     }
   }
   __syncthreads();
-  for (int i = tid; i < ntok * pl.M; i += kUpdThreads) {
-    const int t = i / pl.M, m = i - t * pl.M;
+  // one byte per code, or two 4-bit codes per byte (subspace 2j in the low nibble of byte j)
+  for (int i = tid; i < ntok * pl.code_bytes; i += kUpdThreads) {
+    const int t = i / pl.code_bytes, j = i - t * pl.code_bytes;
     const int pos = p0 + t;
-    if (pos >= 0 && pos < pl.N_max) codes[(ukv * pl.N_max + pos) * pl.M + m] = s_code[t][m];
+    const uint8_t byte = pl.n_code == 16 ? (uint8_t)(s_code[t][2 * j] | (s_code[t][2 * j + 1] << 4))
+                                         : s_code[t][j];
+    if (pos >= 0 && pos < pl.N_max) codes[(ukv * pl.N_max + pos) * pl.code_bytes + j] = byte;
   }
 }
 

@@ -34,7 +34,8 @@ class IvfPqIndex:
     """Index arrays in the layout the C ABI documents (all on one device)."""
     centroids: torch.Tensor     # [B, Hkv, n_list, d]        f32
     codebooks: torch.Tensor     # [B, Hkv, M, 256, dsub]     f32
-    codes: torch.Tensor         # [B, Hkv, N_max, M]         u8
+    codes: torch.Tensor         # [B, Hkv, N_max, M] u8, or [.., M / 2] with two 4-bit codes per
+                                # byte (subspace 2j in the low nibble) when pq_ncode == 16
     list_ids: torch.Tensor      # [B, Hkv, N_max]            int16 storage of uint16 ids
     key_norms: torch.Tensor     # [B, Hkv, N_max]            f32
     list_vmeans: torch.Tensor   # [B, Hkv, n_list, d]        f32
@@ -122,7 +123,7 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
     out = IvfPqIndex(
         torch.zeros((B, Hkv, nl, d), dtype=torch.float32, device=dev),
         torch.zeros((B, Hkv, M, nc, dsub), dtype=torch.float32, device=dev),
-        torch.zeros((B, Hkv, Nmax, M), dtype=torch.uint8, device=dev),
+        torch.zeros((B, Hkv, Nmax, M if nc > 16 else M // 2), dtype=torch.uint8, device=dev),
         torch.zeros((B, Hkv, Nmax), dtype=torch.int16, device=dev),
         torch.zeros((B, Hkv, Nmax), dtype=torch.float32, device=dev),
         torch.zeros((B, Hkv, nl, d), dtype=torch.float32, device=dev),
@@ -160,7 +161,8 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
                                 torch.zeros_like(vsum))
             out.centroids[b, g] = c
             out.codebooks[b, g] = cb
-            out.codes[b, g, :n] = codes.T.to(torch.uint8)
+            ct = codes.T.to(torch.uint8)                          # [n, M]
+            out.codes[b, g, :n] = ct if nc > 16 else (ct[:, 0::2] | (ct[:, 1::2] << 4))
             out.list_ids[b, g, :n] = ids.to(torch.int16)
             out.key_norms[b, g, :n] = r
             out.list_vmeans[b, g] = vmean.float()

@@ -41,7 +41,7 @@ class DecodeOp:
             batch=cfg.batch, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
             n_list=cfg.n_list, pq_m=cfg.pq_m, max_seq_len=self.codes.shape[2],
             max_pages_per_seq=inp.max_pages_per_seq, budget_ppm=ppm, dtype=cfg.dtype,
-            head_dim=cfg.head_dim, page_size=cfg.page_size, n_sink=cfg.n_sink,
+            head_dim=cfg.head_dim, pq_ncode=cfg.pq_ncode, page_size=cfg.page_size, n_sink=cfg.n_sink,
             n_local=cfg.n_local, exact_set_multiple=cfg.exact_set_multiple)
         self.index = pqhsa.make_index(self.centroids, self.codebooks, self.codes, self.list_ids,
                                       self.key_norms, self.list_vmeans)

@@ -84,6 +84,11 @@ def named_config(name: str) -> DecodeConfig:
         return DecodeConfig("c1", 1, 4, 1, (4096,), "fp16", 64, 16, 20000, seed=0)
     if name == "c2":       # Llama-3.1-8B-shaped layer, 32K
         return DecodeConfig("c2", 1, 32, 8, (32 * K,), "bf16", 256, 32, 20000, seed=2000)
+    if name.startswith("c3p"):  # c3p_b{B}_r{pct}: the same layer in the paper's own index setting
+        _, b, r = name.split("_")  # (512 lists, 8 subspaces of 4 bits, 4 sinks, 128-token window,
+        batch, pct = int(b[1:]), int(r[1:])          # exact set in whole pages; App. A)
+        return DecodeConfig(name, batch, 32, 8, (128 * K,) * batch, "bf16", 512, 8, pct * 10000,
+                            seed=3000, pq_ncode=16, n_sink=4, n_local=128, exact_set_multiple=16)
     if name.startswith("c3"):   # c3_b{1,8}_r{1,2}: Llama-3.1-8B-shaped layer, 128K
         _, b, r = name.split("_")
         batch, pct = int(b[1:]), int(r[1:])

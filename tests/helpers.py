@@ -23,11 +23,23 @@ def oracle_arrays(inp, idx):
     f64 = lambda t: t.detach().cpu().double().numpy()
     a = dict(
         q=f64(inp.q), centroids=f64(idx.centroids), codebooks=f64(idx.codebooks),
-        codes=idx.codes.cpu().numpy(), list_ids=idx.list_ids.cpu().numpy().view(np.uint16),
+        codes=unpacked_codes(idx.codes.cpu().numpy(), inp.cfg),
+        list_ids=idx.list_ids.cpu().numpy().view(np.uint16),
         key_norms=f64(idx.key_norms), list_vmeans=f64(idx.list_vmeans),
         k_cache_flat=f64(inp.k_cache.reshape(-1)), v_cache_flat=f64(inp.v_cache.reshape(-1)),
         block_table=inp.block_table.cpu().numpy(), seq_lens=inp.seq_lens.cpu().numpy())
     return a
+
+
+def unpacked_codes(codes: np.ndarray, cfg) -> np.ndarray:
+    """One code per byte for the oracle: 4-bit indices come two per byte (subspace 2j in the low
+    nibble of byte j)."""
+    if cfg.pq_ncode > 16:
+        return codes
+    out = np.empty(codes.shape[:-1] + (cfg.pq_m,), dtype=np.uint8)
+    out[..., 0::2] = codes & 15
+    out[..., 1::2] = codes >> 4
+    return out
 
 
 def oracle_arrays_for_sequence(inp, idx, b):
@@ -43,7 +55,8 @@ def oracle_arrays_for_sequence(inp, idx, b):
     sl = slice(b, b + 1)
     return dict(
         q=f64(inp.q[sl]), centroids=f64(idx.centroids[sl]), codebooks=f64(idx.codebooks[sl]),
-        codes=idx.codes[sl].cpu().numpy(), list_ids=idx.list_ids[sl].cpu().numpy().view(np.uint16),
+        codes=unpacked_codes(idx.codes[sl].cpu().numpy(), cfg),
+        list_ids=idx.list_ids[sl].cpu().numpy().view(np.uint16),
         key_norms=f64(idx.key_norms[sl]), list_vmeans=f64(idx.list_vmeans[sl]),
         k_cache_flat=f64(inp.k_cache[pages].reshape(-1)),
         v_cache_flat=f64(inp.v_cache[pages].reshape(-1)),

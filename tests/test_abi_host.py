@@ -73,6 +73,8 @@ def test_group_of_eight_is_two_head_groups_and_padded_groups():
     (dict(exact_set_multiple=16, k_max=1311), pqhsa.ERR_INVALID_ARG),   # no room for the rounding
     (dict(head_dim=64, pq_m=16), pqhsa.ERR_UNSUPPORTED),
     (dict(pq_m=4), pqhsa.ERR_UNSUPPORTED),
+    (dict(pq_ncode=16, pq_m=32), pqhsa.ERR_UNSUPPORTED),  # 4-bit codes: 8 or 16 subspaces
+    (dict(pq_ncode=64), pqhsa.ERR_UNSUPPORTED),
     (dict(n_list=8192), pqhsa.ERR_UNSUPPORTED),
     (dict(max_seq_len=131070), pqhsa.ERR_UNSUPPORTED),
     (dict(n_q_heads=30), pqhsa.ERR_INVALID_ARG),          # not a multiple of n_kv_heads

@@ -30,6 +30,8 @@ CASES = [
     # the paper's own partition at 128K: 4 sinks, 128-token window, exact set in whole pages
     # (1,456 tokens at 1 %, App. A)
     ("c3_b1_r1+sinks_window_pages", [(0, 2), (0, 27)]),
+    # ... and with the paper's own index on top: 512 lists, eight 4-bit subspaces
+    ("c3p_b1_r1", [(0, 6), (0, 21)]),
 ]
 
 

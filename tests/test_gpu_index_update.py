@@ -15,7 +15,7 @@ from paper_2609_33746_b200 import pqhsa
 from paper_2609_33746_b200.runner import DecodeOp
 from paper_2609_33746_b200.workload import DecodeConfig
 
-from helpers import make_case
+from helpers import make_case, unpacked_codes
 
 pytestmark = pytest.mark.gpu
 
@@ -36,6 +36,7 @@ CASES = {
     "m8_many_lists_one_empty_update": (cfg_of("u3", pq_m=8, n_list=256, seq_lens=(4000, 1200)),
                                        (300, 0)),
     "m64": (cfg_of("u4", pq_m=64, batch=1, seq_lens=(1500,)), (129,)),
+    "four_bit_m8": (cfg_of("u7", pq_m=8, pq_ncode=16, n_list=128, seq_lens=(2500, 800)), (256, 77)),
 }
 
 
@@ -80,12 +81,13 @@ def test_index_update_matches_oracle(key):
             lo, hi = first[b], cfg.seq_lens[b]
             ref = O.index_update(
                 idx.centroids[b, g].cpu().double().numpy(), idx.codebooks[b, g].cpu().double().numpy(),
-                want_codes[b, g].cpu().numpy() * 0, np.zeros(want_ids.shape[2], dtype=np.uint16),
+                np.zeros((want_ids.shape[2], cfg.pq_m), dtype=np.uint8),
+                np.zeros(want_ids.shape[2], dtype=np.uint16),
                 np.zeros(want_ids.shape[2]), vm0[b, g].cpu().double().numpy(),
                 cnt0[b, g].cpu().numpy(), k[lo:hi].cpu().double().numpy(),
                 v[lo:hi].cpu().double().numpy(), first_pos=lo)
             got_ids = (idx.list_ids[b, g, lo:hi].cpu().numpy().view(np.uint16)).astype(np.int64)
-            got_codes = idx.codes[b, g, lo:hi].cpu().numpy().astype(np.int64)
+            got_codes = unpacked_codes(idx.codes[b, g, lo:hi].cpu().numpy(), cfg).astype(np.int64)
             got_norms = idx.key_norms[b, g, lo:hi].cpu().double().numpy()
             np.testing.assert_allclose(got_norms, ref["key_norms"][lo:hi], rtol=2e-6)
             want_a = ref["list_ids"][lo:hi].astype(np.int64)

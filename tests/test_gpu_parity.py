@@ -78,6 +78,14 @@ CASES = {
     # the largest list count, most lists empty
     "lists_4096_mostly_empty": small("l4096", seq_lens=(3000,), n_list=4096, n_q_heads=4,
                                      n_kv_heads=1, kmeans_iters=1),
+    # the paper's own index setting: eight 16-dim subspaces of four bits (two codes per byte,
+    # 4 bytes of codes per token), 512 lists, 4 sinks, 128-token window, page-rounded budget
+    "paper_index_4bit": small("p4", pq_m=8, pq_ncode=16, n_list=512, seq_lens=(6000,), n_sink=4,
+                              n_local=128, exact_set_multiple=16, kmeans_iters=2),
+    "four_bit_m16_g2_ragged": small("p4b", pq_m=16, pq_ncode=16, batch=3, seq_lens=(2100, 0, 333),
+                                    n_q_heads=4, n_kv_heads=2),
+    "four_bit_g1_fp16": small("p4c", pq_m=8, pq_ncode=16, n_q_heads=2, n_kv_heads=2, dtype="fp16",
+                              seq_lens=(1500,)),
 }
 
 
@@ -120,7 +128,7 @@ def test_stage_lut(key):
     torch.cuda.synchronize()
     Gc = pqhsa.heads_per_group(op.params)
     n_hg = (cfg.group + Gc - 1) // Gc
-    lut = op.lut.view(cfg.batch, cfg.n_kv_heads, n_hg, 256, cfg.pq_m, Gc).cpu().double().numpy()
+    lut = op.lut.view(cfg.batch, cfg.n_kv_heads, n_hg, cfg.pq_ncode, cfg.pq_m, Gc).cpu().double().numpy()
     coarse = op.coarse.view(cfg.batch, cfg.n_kv_heads, n_hg, cfg.n_list, Gc).cpu().double().numpy()
     for (b, h), r in ref.items():
         kv, hh = divmod(h, cfg.group)
@@ -132,7 +140,7 @@ def test_stage_lut(key):
         assert np.abs(coarse[b, kv, hg, :, g] - want_coarse).max() <= 1e-5 * scale
     # padded head slots are zero
     if n_hg * Gc > cfg.group:
-        assert float(op.lut.view(cfg.batch, cfg.n_kv_heads, n_hg, 256, cfg.pq_m, Gc)
+        assert float(op.lut.view(cfg.batch, cfg.n_kv_heads, n_hg, cfg.pq_ncode, cfg.pq_m, Gc)
                      [:, :, -1, :, :, cfg.group - (n_hg - 1) * Gc:].abs().max()) == 0.0
 
 

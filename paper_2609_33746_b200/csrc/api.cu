@@ -78,9 +78,11 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.k_max = p->k_max; o.n_sink = p->n_sink; o.n_local = p->n_local;
   o.exact_multiple = p->exact_set_multiple; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
   o.num_sms = sm_count();
-  o.scan_ctas = o.num_sms;
+  // persistent scan CTAs: one per SM, two with the small tables of 4-bit codes
+  o.scan_ctas = o.n_code == 16 ? 2 * o.num_sms : o.num_sms;
   o.upb = o.Hkv * o.n_hg;
   o.n_part = o.scan_ctas / o.upb + 2;
+  if (o.n_part > kMaxSeg) return PQHSA_ERR_UNSUPPORTED;     // more SMs than this build plans for
   o.rows = o.B * o.Hq;
   // the coarse table is bulk-copied: its byte size and unit stride must be multiples of 16.
   // Prefer a 3-stage code ring with the coarse table in shared memory, then give up the

@@ -18,7 +18,6 @@ namespace pqhsa {
 namespace {
 
 constexpr int kBgThreads = 128;
-constexpr int kMaxSeg = 160;                  // >= n_part for any plan (148 SMs / 1 unit + 2)
 
 // grid (bg_ctas, rows).  CTA c merges a slice of the lists and subtracts a slice of the
 // selected tokens; both go into bg_mass (zeroed by the caller) with float atomics, so the
@@ -73,7 +72,8 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   const int nseg = min(kMaxSeg, split_cta_of(sp, s_u + tb - 1) - c_first + 1);
   const float* pr = partials + (size_t)row * pl.n_part * (n_list + 1);
 
-  if (tid < nseg) s_scale[tid] = pr[(size_t)tid * (n_list + 1)];     // segment maxima
+  for (int sg = tid; sg < nseg; sg += kBgThreads)                      // segment maxima
+    s_scale[sg] = pr[(size_t)sg * (n_list + 1)];
   __syncthreads();
   float m = -CUDART_INF_F;
   for (int s = 0; s < nseg; ++s) m = fmaxf(m, s_scale[s]);
@@ -83,7 +83,8 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   }
   const float m2 = m * kLog2e;
   __syncthreads();
-  if (tid < nseg) s_scale[tid] = fast_exp2(fmaf(s_scale[tid], kLog2e, -m2));
+  for (int sg = tid; sg < nseg; sg += kBgThreads)
+    s_scale[sg] = fast_exp2(fmaf(s_scale[sg], kLog2e, -m2));
   __syncthreads();
   const int jl = (int)((long long)c * n_list / C), jh = (int)((long long)(c + 1) * n_list / C);
   for (int j = jl + tid; j < jh; j += kBgThreads) {

@@ -19,6 +19,7 @@ constexpr int kTile = 32;            // tokens per scan tile: one token per lane
 #endif
 constexpr int kScanThreads = PQHSA_SCAN_THREADS;
 constexpr int kScanMinTiles = kScanThreads / 32;   // a scan CTA gets at least one tile per warp
+constexpr int kMaxSeg = 320;                       // scan segments one unit may be cut into (n_part)
 constexpr int kHistBins = 4096;      // 12-bit radix digits of the select's shared-memory histograms
 constexpr int kSelThreads = 512;
 constexpr int kSelChunk = 8192;      // scores per select CTA: 16 per thread, kept in registers

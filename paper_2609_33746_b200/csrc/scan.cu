@@ -196,7 +196,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
 // kBits = 8: one byte per code, 256-entry tables.  kBits = 4: two codes per byte (subspace 2j in
 // the low nibble of byte j), 16-entry tables.
 template <int M, int GC, int kStages, int kBits>
-__global__ void __launch_bounds__(kScanThreads, 1)
+__global__ void __launch_bounds__(kScanThreads, kBits == 4 ? 2 : 1)
 scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restrict__ lids,
             const float* __restrict__ norms, const float* __restrict__ lut,
             const float* __restrict__ coarse, const int32_t* __restrict__ seq_lens,

@@ -86,6 +86,13 @@ CASES = {
                                     n_q_heads=4, n_kv_heads=2),
     "four_bit_g1_fp16": small("p4c", pq_m=8, pq_ncode=16, n_q_heads=2, n_kv_heads=2, dtype="fp16",
                               seq_lens=(1500,)),
+    # one (sequence, KV head, head group) cut into as many scan segments as there are scan CTAs
+    # (two per SM with 4-bit codes): the most list partials a row can have
+    "four_bit_single_unit_all_ctas": small("p4d", pq_m=8, pq_ncode=16, n_q_heads=4, n_kv_heads=1,
+                                           seq_lens=(160000,), n_list=128, kmeans_iters=1,
+                                           budget_ppm=5000),
+    "single_unit_all_ctas": small("u1", n_q_heads=4, n_kv_heads=1, seq_lens=(80000,), n_list=128,
+                                  kmeans_iters=1, budget_ppm=5000),
 }
 
 

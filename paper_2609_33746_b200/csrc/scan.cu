@@ -386,11 +386,12 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         if (valid) {
           // sink and window tokens are attended exactly: their score is -inf, so that the
           // top-k never picks them and they add nothing to the list sums
+          float* srow = scores + (size_t)row0 * N_max + i;      // row of head 0; heads N_max apart
 #pragma unroll
           for (int g = 0; g < GC; ++g) {
             if (g < n_heads) {
               if (in_r) sc[g] = cur.norm * (co[g] + accf[g]);
-              scores[(size_t)(row0 + g) * N_max + i] = sc[g];
+              srow[g * N_max] = sc[g];
               mx[g] = fmaxf(mx[g], sc[g]);
             }
           }

@@ -53,11 +53,17 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--kmeans-iters", type=int, default=2)
+    ap.add_argument("--paper-index", action="store_true",
+                    help="the paper's own index setting: 512 lists, 8 subspaces of 4 bits, 4 sinks, "
+                         "128-token window, exact set in whole pages")
     args = ap.parse_args()
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     for ctx in (int(x) for x in args.contexts.split(",")):
         cfg = dataclasses.replace(named_config(f"c5_n{ctx}_b{args.batch}"),
                                   kmeans_iters=args.kmeans_iters)
+        if args.paper_index:
+            cfg = dataclasses.replace(cfg, n_list=512, pq_m=8, pq_ncode=16, n_sink=4, n_local=128,
+                                      exact_set_multiple=16)
         inp = generate(cfg, device="cuda")
         idx = build_index(inp)
         op = DecodeOp(inp, idx)

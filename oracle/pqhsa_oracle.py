@@ -20,6 +20,8 @@ re-ordering:
     O9  y^ = (N_E + N^_B) / (Z_E + Z^_B)                                 (Eq. 5)
     O10 index maintenance: new tokens encoded into the existing lists,  (Sec. 3.3, first paragraph;
         list means refreshed, no re-clustering                           Sec. 3.1 for the encoding)
+    V   the mechanism variants T, Bx, C, C2, C2b: other ways to form     (Table 2; App. B, "Variant
+        the background term, same selector, budget and exact part        definitions")
 
 Readings where the paper is silent (the repository's design notes list them too):
   * top-k ties: stable, the lower position wins;
@@ -28,6 +30,12 @@ Readings where the paper is silent (the repository's design notes list them too)
   * the list mean that multiplies M_j is the stored mean over all members of the
     list, selected ones included (Sec. 3.2, last paragraph);
   * an empty list contributes zero (text after Eq. 4);
+  * the window L holds whatever the index does not cover yet: with `indexed_len` given,
+    R = [|S|, indexed_len) and L = [indexed_len, N) (Sec. 3.3: new tokens stay exact until
+    the next periodic update), otherwise L is the last n_local tokens;
+  * variants: |R_j| is counted from the list ids of R; with an empty T the shared logit of
+    C2 / C2b does not exist and the background is dropped; a list with no unselected member
+    has no Bx mean and no mass;
   * index maintenance: a new key goes to the list whose centroid is nearest to its direction
     in squared Euclidean distance (the assignment rule of k-means, the lower index on ties),
     each sub-vector of the residual to its nearest codeword likewise, a zero key has
@@ -38,9 +46,12 @@ against a dense dot product with the reconstructed key, rho = 1 against textbook
 softmax attention, the exact-reconstruction / constant-value-per-list case against
 textbook attention at any budget, a hand-computed closed form, mass conservation,
 shift and permutation invariance, the budgets the paper prints (1,456 and 2,752
-tokens at 131,072), and top-k against a full sort; for O10 scalar-loop brute force, the
-from-scratch mean of all members, a key on a centroid, and one update against two.  No
-function here is "parity unpinned".
+tokens at 131,072, also as the k that decode_head selects there), and top-k against a full
+sort; decode() (query head -> KV head map, paged reads through two stride layouts) against
+scalar loops on dense per-head arrays; for O10 scalar-loop brute force, the from-scratch mean
+of all members, a key on a centroid, and one update against two; for the variants scalar loops,
+hand-computed closed forms (2.125 / 2.5 / 1) and the cases where two variants must coincide.
+No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -58,11 +69,19 @@ def budget_k(n_indexed: int, budget_ppm: int) -> int:
     return min(k, n_indexed)
 
 
-def partition(seq_len: int, n_sink: int = 0, n_local: int = 0):
+def partition(seq_len: int, n_sink: int = 0, n_local: int = 0, indexed_len=None):
     """Sink prefix S, local window L (most recent tokens) and indexed region R
-    (Sec. 3.2).  Returned as position arrays; they are disjoint and cover [0, N)."""
+    (Sec. 3.2).  Returned as position arrays; they are disjoint and cover [0, N).
+
+    The window holds the tokens that are not in the index yet (Sec. 3.3: a new token is
+    attended exactly until the next periodic update encodes it).  `indexed_len` is the
+    number of leading positions the index covers, so R = [|S|, indexed_len) and L is
+    everything after; without it the window is the last n_local tokens."""
     n_s = min(n_sink, seq_len)
-    l_start = max(n_s, seq_len - n_local)
+    if indexed_len is None:
+        l_start = max(n_s, seq_len - n_local)
+    else:
+        l_start = min(seq_len, max(n_s, int(indexed_len)))
     S = np.arange(0, n_s, dtype=np.int64)
     R = np.arange(n_s, l_start, dtype=np.int64)
     L = np.arange(l_start, seq_len, dtype=np.int64)
@@ -70,10 +89,10 @@ def partition(seq_len: int, n_sink: int = 0, n_local: int = 0):
 
 
 def exact_set_tokens(seq_len: int, n_sink: int, n_local: int, budget_ppm: int,
-                     round_to_page: int = 0) -> int:
+                     round_to_page: int = 0, indexed_len=None) -> int:
     """Number of tokens attended exactly: |S| + |L| + ceil(rho |R|), optionally
     rounded up to whole pages (App. A, "Budgets")."""
-    S, L, R = partition(seq_len, n_sink, n_local)
+    S, L, R = partition(seq_len, n_sink, n_local, indexed_len)
     total = len(S) + len(L) + budget_k(len(R), budget_ppm)
     if round_to_page:
         total = round_to_page * ((total + round_to_page - 1) // round_to_page)
@@ -146,24 +165,61 @@ def gather_rows(cache_flat: np.ndarray, block_table_row: np.ndarray, positions: 
 
 
 # --------------------------------------------------------------------------- O6-O9
+VARIANTS = ("B", "T", "Bx", "C", "C2", "C2b")
+
+
 def hybrid_output(q: np.ndarray, keys_E: np.ndarray, vals_E: np.ndarray,
                   logits_B: np.ndarray, lists_B: np.ndarray, list_vmeans: np.ndarray,
-                  sm_scale: float):
+                  sm_scale: float, variant: str = "B", list_counts=None, is_T=None,
+                  lists_T=None, approx_T=None):
     """Eq. 4-5 for one query head.
 
     keys_E, vals_E: original rows of the exact set E.  logits_B, lists_B: the
     approximate logit and list id of every background token (B = R \\ T).
     list_vmeans [n_list, d]: stored per-list value means.
-    Returns y^ and a dict with the intermediate sums (all relative to m_0)."""
+    Returns y^ and a dict with the intermediate sums (all relative to m_0).
+
+    `variant` switches how the background term is formed (Table 2 and App. B, "Variant
+    definitions"); selector, budget and exact part are the same in all of them:
+      B    PQ-HSA itself: logit l~_i, value vbar_j                               (Eq. 4)
+      T    no background term (its logits are -inf)
+      Bx   B with vbar_j replaced by the mean over the list's UNSELECTED members,
+           (|R_j| vbar_j - sum_{i in T n R_j} v_i) / |B n R_j|
+      C    logit l~_i, value = the token-count-weighted global mean
+           vbar_global = sum_j |R_j| vbar_j / sum_j |R_j|
+      C2   one shared logit mean_{i in T} l~_i for every background token, vbar_global
+      C2b  one shared logit min_{i in T} l_i (exact logits), vbar_global
+    The variants other than B and T need list_counts [n_list] = |R_j|; Bx also needs
+    is_T (bool over the rows of E) and lists_T (list id of each selected row, in the
+    order they appear in E); C2 needs approx_T (l~_i of the selected rows).
+    Reading: with an empty T the shared logit of C2 / C2b is undefined and the background
+    is dropped; a list whose members are all selected has no unselected mean and no mass."""
+    if variant not in VARIANTS:
+        raise ValueError(variant)
     q = np.asarray(q, dtype=np.float64)
     d = q.shape[0]
     list_vmeans = np.asarray(list_vmeans, dtype=np.float64)
     n_list = list_vmeans.shape[0]
     logits_E = (np.asarray(keys_E, dtype=np.float64).reshape(-1, d) @ q) * sm_scale
+    vals_E = np.asarray(vals_E, dtype=np.float64).reshape(-1, d)
     logits_B = np.asarray(logits_B, dtype=np.float64)
     lists_B = np.asarray(lists_B).astype(np.int64)
 
+    # background logits of the variant
+    if variant == "T":
+        logits_B = np.full(logits_B.shape, -math.inf)
+    elif variant in ("C2", "C2b"):
+        n_T = 0 if is_T is None else int(np.count_nonzero(is_T))
+        if n_T == 0:
+            shared = -math.inf
+        elif variant == "C2":
+            shared = float(np.mean(np.asarray(approx_T, dtype=np.float64)))
+        else:
+            shared = float(np.min(logits_E[np.asarray(is_T, dtype=bool)]))
+        logits_B = np.full(logits_B.shape, shared)
+
     cands = [x.max() for x in (logits_E, logits_B) if x.size]
+    cands = [c for c in cands if c > -math.inf]
     if not cands:                                   # empty sequence
         return np.zeros(d), dict(m0=-math.inf, Z_E=0.0, Z_B=0.0, M=np.zeros(n_list),
                                  logits_E=logits_E)
@@ -171,11 +227,30 @@ def hybrid_output(q: np.ndarray, keys_E: np.ndarray, vals_E: np.ndarray,
     e_E = np.exp(logits_E - m0)
     e_B = np.exp(logits_B - m0)
     Z_E = e_E.sum()
-    N_E = e_E @ np.asarray(vals_E, dtype=np.float64).reshape(-1, d)
+    N_E = e_E @ vals_E
     # M_j = sum of e~_i over the background members of list j (empty list -> 0)
     M_j = np.bincount(lists_B, weights=e_B, minlength=n_list).astype(np.float64)
     Z_B = M_j.sum()
-    N_B = M_j @ list_vmeans
+
+    # background values of the variant
+    if variant in ("B", "T"):
+        N_B = M_j @ list_vmeans
+    elif variant == "Bx":
+        counts = np.asarray(list_counts, dtype=np.float64)
+        sel_rows = vals_E[np.asarray(is_T, dtype=bool)]
+        sel_lists = np.asarray(lists_T).astype(np.int64)
+        sum_T = np.zeros((n_list, d))
+        np.add.at(sum_T, sel_lists, sel_rows)
+        n_unsel = counts - np.bincount(sel_lists, minlength=n_list)
+        vbar_B = np.zeros((n_list, d))
+        has = n_unsel > 0
+        vbar_B[has] = (counts[has, None] * list_vmeans[has] - sum_T[has]) / n_unsel[has, None]
+        N_B = M_j @ vbar_B
+    else:                                            # C, C2, C2b
+        counts = np.asarray(list_counts, dtype=np.float64)
+        total = counts.sum()
+        v_global = (counts @ list_vmeans) / total if total > 0 else np.zeros(d)
+        N_B = Z_B * v_global
     y = (N_E + N_B) / (Z_E + Z_B)
     return y, dict(m0=m0, Z_E=Z_E, Z_B=Z_B, M=M_j, logits_E=logits_E,
                    lse=m0 + math.log(Z_E + Z_B))
@@ -183,30 +258,35 @@ def hybrid_output(q: np.ndarray, keys_E: np.ndarray, vals_E: np.ndarray,
 
 def decode_head(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
                 keys, vals, seq_len, budget_ppm, sm_scale, n_sink=0, n_local=0,
-                round_exact_set_to_page=0):
+                round_exact_set_to_page=0, indexed_len=None, variant="B"):
     """One (sequence, query head): O1-O9.
 
     keys / vals are callables position-array -> rows [len, d] (original K, V of the
     query head's KV head); the index arrays belong to the same KV head and are
     indexed by sequence position.  Returns a dict with y^ and every intermediate."""
     q = np.asarray(q, dtype=np.float64)
-    S, L, R = partition(seq_len, n_sink, n_local)
+    S, L, R = partition(seq_len, n_sink, n_local, indexed_len)
     k = budget_k(len(R), budget_ppm)
     if round_exact_set_to_page:
-        total = exact_set_tokens(seq_len, n_sink, n_local, budget_ppm, round_exact_set_to_page)
+        total = exact_set_tokens(seq_len, n_sink, n_local, budget_ppm, round_exact_set_to_page,
+                                 indexed_len)
         k = min(len(R), total - len(S) - len(L))
     r_q, u_q = split_query(q)
     coarse, lut = build_lut(u_q, centroids, codebooks)
     norms_R = None if key_norms is None else np.asarray(key_norms)[R]
-    approx = adc_logits(r_q, coarse, lut, np.asarray(codes)[R], np.asarray(list_ids)[R],
-                        norms_R, sm_scale)
+    lists_R = np.asarray(list_ids)[R].astype(np.int64)
+    approx = adc_logits(r_q, coarse, lut, np.asarray(codes)[R], lists_R, norms_R, sm_scale)
     sel_local = select_topk(approx, k)
     T = R[sel_local]
     mask_B = np.ones(len(R), dtype=bool)
     mask_B[sel_local] = False
     E = np.concatenate([S, L, T])
-    y, aux = hybrid_output(q, keys(E), vals(E), approx[mask_B],
-                           np.asarray(list_ids)[R][mask_B], list_vmeans, sm_scale)
+    is_T = np.concatenate([np.zeros(len(S) + len(L), dtype=bool), np.ones(len(T), dtype=bool)])
+    n_list = np.asarray(list_vmeans).shape[0]
+    y, aux = hybrid_output(q, keys(E), vals(E), approx[mask_B], lists_R[mask_B], list_vmeans,
+                           sm_scale, variant=variant,
+                           list_counts=np.bincount(lists_R, minlength=n_list), is_T=is_T,
+                           lists_T=lists_R[sel_local], approx_T=approx[sel_local])
     kth = float(np.sort(approx)[::-1][k - 1]) if k > 0 else math.nan
     aux.update(y=y, r_q=r_q, u_q=u_q, coarse=coarse, lut=lut, approx=approx, R=R, T=T,
                E=E, k=k, kth_score=kth)
@@ -216,11 +296,14 @@ def decode_head(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans
 def decode(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
            k_cache_flat, v_cache_flat, block_table, seq_lens, *, n_kv_heads, page_size,
            stride_page, stride_token, stride_head, budget_ppm, sm_scale,
-           n_sink=0, n_local=0, heads=None, batch_items=None, round_exact_set_to_page=0):
+           n_sink=0, n_local=0, heads=None, batch_items=None, round_exact_set_to_page=0,
+           indexed_lens=None, variant="B"):
     """The whole operator: every (sequence, query head), reading the paged cache in
     place.  Array layouts are those of the C ABI (q [B,Hq,d]; centroids
     [B,Hkv,n_list,d]; codebooks [B,Hkv,M,n_code,dsub]; codes [B,Hkv,N_max,M];
-    list_ids / key_norms [B,Hkv,N_max]; list_vmeans [B,Hkv,n_list,d]).
+    list_ids / key_norms [B,Hkv,N_max]; list_vmeans [B,Hkv,n_list,d]).  Query head h reads
+    the index and the cache rows of KV head h // G, G = Hq / n_kv_heads (Sec. 3.3: the heads
+    of a group share their KV head's codes).  indexed_lens [B] (optional): see partition().
     Returns {(b, h): decode_head result}; `heads` / `batch_items` restrict the work."""
     q = np.asarray(q, dtype=np.float64)
     B, Hq, d = q.shape
@@ -239,7 +322,8 @@ def decode(q, centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
             out[(b, h)] = decode_head(
                 q[b, h], centroids[b, g], codebooks[b, g], codes[b, g], list_ids[b, g],
                 None if key_norms is None else key_norms[b, g], list_vmeans[b, g],
-                keys, vals, n, budget_ppm, sm_scale, n_sink, n_local, round_exact_set_to_page)
+                keys, vals, n, budget_ppm, sm_scale, n_sink, n_local, round_exact_set_to_page,
+                None if indexed_lens is None else int(indexed_lens[b]), variant)
     return out
 
 

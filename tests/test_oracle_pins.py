@@ -397,3 +397,262 @@ def test_index_update_in_two_steps_equals_one_step():
     assert np.array_equal(one["list_counts"], b["list_counts"])
     np.testing.assert_allclose(one["list_vmeans"], b["list_vmeans"], atol=1e-12)
     np.testing.assert_allclose(one["key_norms"], b["key_norms"], atol=0)
+
+
+# ----------------------------------------------------------------------------- decode(): GQA map and paged glue
+def _paged_case(rng, layout, B=2, Hkv=2, G=2, d=4, P=4, n_list=3, M=2, n_code=4,
+                seq_lens=(21, 10)):
+    """A tiny batch in the C ABI's layouts with a shuffled block table.  Returns the arrays
+    decode() takes plus dense per-(sequence, KV head) copies K[b][g], V[b][g] for brute force."""
+    Hq, dsub = Hkv * G, d // M
+    N_max = max(seq_lens)
+    pages = [(n + P - 1) // P for n in seq_lens]
+    total = sum(pages) + 2                                   # two pages nobody owns
+    perm = rng.permutation(total)
+    table = np.zeros((B, max(pages)), dtype=np.int32)
+    o = 0
+    for b in range(B):
+        table[b, :pages[b]] = perm[o:o + pages[b]]
+        o += pages[b]
+    K = rng.normal(size=(B, Hkv, N_max, d))
+    V = rng.normal(size=(B, Hkv, N_max, d))
+    if layout == "split":
+        kc = np.full((total, P, Hkv, d), 99.0)
+        vc = np.full((total, P, Hkv, d), -99.0)
+        strides = (P * Hkv * d, Hkv * d, d)
+        for b in range(B):
+            for i in range(seq_lens[b]):
+                kc[table[b, i // P], i % P] = K[b, :, i]
+                vc[table[b, i // P], i % P] = V[b, :, i]
+        k_flat, v_flat = kc.ravel(), vc.ravel()
+    else:
+        buf = np.full((total, Hkv, P, 2 * d), 99.0)
+        strides = (Hkv * P * 2 * d, 2 * d, P * 2 * d)
+        for b in range(B):
+            for i in range(seq_lens[b]):
+                buf[table[b, i // P], :, i % P, :d] = K[b, :, i]
+                buf[table[b, i // P], :, i % P, d:] = V[b, :, i]
+        k_flat, v_flat = buf.ravel(), buf.ravel()[d:]
+    arrays = dict(
+        q=rng.normal(size=(B, Hq, d)),
+        centroids=rng.normal(size=(B, Hkv, n_list, d)) * 0.3,
+        codebooks=rng.normal(size=(B, Hkv, M, n_code, dsub)) * 0.1,
+        codes=rng.integers(0, n_code, (B, Hkv, N_max, M)).astype(np.uint8),
+        list_ids=rng.integers(0, n_list, (B, Hkv, N_max)).astype(np.uint16),
+        key_norms=rng.uniform(0.5, 2.0, (B, Hkv, N_max)),
+        list_vmeans=rng.normal(size=(B, Hkv, n_list, d)),
+        k_cache_flat=k_flat, v_cache_flat=v_flat, block_table=table,
+        seq_lens=np.array(seq_lens, dtype=np.int32))
+    return arrays, strides, K, V, dict(B=B, Hkv=Hkv, G=G, Hq=Hq, d=d, P=P)
+
+
+@pytest.mark.parametrize("layout", ["split", "interleaved"])
+def test_decode_maps_query_heads_to_kv_heads_and_reads_pages_in_place(layout):
+    """decode() against scalar loops that choose the KV head floor(h / G) themselves and are
+    handed dense K, V (Sec. 3.3: the query heads of a group share their KV head's codes; App. E:
+    rows are read from the engine's pages through strides).  Every (sequence, KV head) has its
+    own index and its own keys, so a wrong head map (h % H_kv, a swapped b/g) or a wrong page
+    lookup changes the result."""
+    rng = np.random.default_rng(21)
+    a, strides, K, V, sh = _paged_case(rng, layout)
+    ppm, n_sink, n_local = 200000, 1, 3
+    res = O.decode(a["q"], a["centroids"], a["codebooks"], a["codes"], a["list_ids"],
+                   a["key_norms"], a["list_vmeans"], a["k_cache_flat"], a["v_cache_flat"],
+                   a["block_table"], a["seq_lens"], n_kv_heads=sh["Hkv"], page_size=sh["P"],
+                   stride_page=strides[0], stride_token=strides[1], stride_head=strides[2],
+                   budget_ppm=ppm, sm_scale=1.0 / math.sqrt(sh["d"]), n_sink=n_sink,
+                   n_local=n_local)
+    assert set(res) == {(b, h) for b in range(sh["B"]) for h in range(sh["Hq"])}
+    for b in range(sh["B"]):
+        n = int(a["seq_lens"][b])
+        for h in range(sh["Hq"]):
+            g = h // sh["G"]
+            y_bf, T_bf, _ = brute_force(a["q"][b, h], a["centroids"][b, g], a["codebooks"][b, g],
+                                        a["codes"][b, g, :n], a["list_ids"][b, g, :n],
+                                        a["key_norms"][b, g, :n], a["list_vmeans"][b, g],
+                                        K[b, g, :n], V[b, g, :n], ppm, n_sink, n_local)
+            assert sorted(res[(b, h)]["T"].tolist()) == T_bf
+            np.testing.assert_allclose(res[(b, h)]["y"], y_bf, rtol=1e-11, atol=1e-13)
+    # the two query heads of a group see the same keys but are different rows
+    assert not np.allclose(res[(0, 0)]["y"], res[(0, 1)]["y"])
+
+
+def test_decode_head_restriction_keeps_absolute_head_numbers():
+    rng = np.random.default_rng(22)
+    a, strides, K, V, sh = _paged_case(rng, "split")
+    kw = dict(n_kv_heads=sh["Hkv"], page_size=sh["P"], stride_page=strides[0],
+              stride_token=strides[1], stride_head=strides[2], budget_ppm=250000,
+              sm_scale=0.5)
+    args = (a["q"], a["centroids"], a["codebooks"], a["codes"], a["list_ids"], a["key_norms"],
+            a["list_vmeans"], a["k_cache_flat"], a["v_cache_flat"], a["block_table"], a["seq_lens"])
+    full = O.decode(*args, **kw)
+    part = O.decode(*args, heads=[3], batch_items=[1], **kw)
+    assert list(part) == [(1, 3)]
+    np.testing.assert_array_equal(part[(1, 3)]["y"], full[(1, 3)]["y"])
+
+
+# ----------------------------------------------------------------------------- page-rounded budget inside decode_head
+@pytest.mark.parametrize("ppm,k_want,tokens", [(10000, 1324, 1456), (20000, 2620, 2752)])
+def test_decode_head_selects_the_page_rounded_budget_at_128k(ppm, k_want, tokens):
+    """App. A, "Budgets": 4 sinks + 128 window tokens + ceil(rho |R|) retrieved tokens, rounded up
+    to pages of 16, are 1,456 / 2,752 tokens at 131,072; decode_head must select exactly the
+    difference (1,324 / 2,620) and report the k-th largest approximate logit."""
+    rng = np.random.default_rng(31)
+    n, d = 131072, 2
+    cen = np.zeros((1, d))
+    cb = rng.normal(size=(1, 256, d))                         # one subspace: the score is LUT[z_i]
+    codes = rng.integers(0, 256, (n, 1)).astype(np.uint8)
+    ids = np.zeros(n, dtype=np.uint16)
+    norms = rng.uniform(0.5, 2.0, n)
+    q = np.array([0.7, -1.1])
+    zeros = lambda pos: np.zeros((len(pos), d))
+    r = O.decode_head(q, cen, cb, codes, ids, norms, np.zeros((1, d)), zeros, zeros, n, ppm,
+                      1.0, n_sink=4, n_local=128, round_exact_set_to_page=16)
+    assert r["k"] == k_want and len(r["T"]) == k_want and len(r["E"]) == tokens
+    assert len(r["R"]) == 130940 and r["T"].min() >= 4 and r["T"].max() < 131072 - 128
+    want = norms[4:n - 128] * (cb[0][codes[4:n - 128, 0]] @ q)       # Eq. 2 with one subspace, c = 0
+    np.testing.assert_allclose(r["approx"], want, rtol=1e-12, atol=1e-14)
+    assert r["kth_score"] == np.sort(r["approx"])[-k_want]
+    assert np.all(r["approx"][r["T"] - 4] >= r["kth_score"])
+    # without rounding the same call takes ceil(rho |R|)
+    r0 = O.decode_head(q, cen, cb, codes, ids, norms, np.zeros((1, d)), zeros, zeros, n, ppm,
+                       1.0, n_sink=4, n_local=128)
+    assert r0["k"] == -(-130940 * ppm // 1_000_000)
+
+
+# ----------------------------------------------------------------------------- window = not yet indexed
+def test_indexed_len_sets_the_window():
+    """Sec. 3.3: tokens written since the last index update stay in the exactly-attended window.
+    partition(indexed_len=r) is the partition with a window of seq_len - r tokens."""
+    for n, n_sink, r_end in [(100, 4, 60), (100, 4, 100), (100, 4, 2), (5, 8, 3), (50, 0, 0)]:
+        S, L, R = O.partition(n, n_sink, 0, indexed_len=r_end)
+        S2, L2, R2 = O.partition(n, n_sink, max(0, n - max(r_end, min(n_sink, n))))
+        assert S.tolist() == S2.tolist() and L.tolist() == L2.tolist() and R.tolist() == R2.tolist()
+        assert sorted(S.tolist() + L.tolist() + R.tolist()) == list(range(n))
+    rng = np.random.default_rng(41)
+    n, d, n_list, M, n_code = 40, 4, 3, 2, 4
+    cen, cb, codes, ids, norms, _ = random_index(rng, n, d, n_list, M, n_code)
+    K, V, q = rng.normal(size=(n, d)), rng.normal(size=(n, d)), rng.normal(size=d)
+    vmeans = rng.normal(size=(n_list, d))
+    a = run_head(q, cen, cb, codes, ids, norms, vmeans, K, V, 200000, n_sink=2, indexed_len=29)
+    y_bf, T_bf, _ = brute_force(q, cen, cb, codes, ids, norms, vmeans, K, V, 200000, 2, n - 29)
+    assert sorted(a["T"].tolist()) == T_bf and a["E"].tolist()[:13] == [0, 1] + list(range(29, 40))
+    np.testing.assert_allclose(a["y"], y_bf, rtol=1e-11, atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- mechanism variants (Table 2, App. B)
+def brute_force_variant(variant, q, cen, cb, codes, ids, norms, vmeans, K, V, ppm):
+    """Scalar loops for the variants of Table 2 (no sinks, no window), from their definitions."""
+    n, d = K.shape
+    M, n_code, dsub = cb.shape
+    n_list = len(vmeans)
+    rq = math.sqrt(sum(float(x) ** 2 for x in q))
+    approx = []
+    for i in range(n):
+        acc = sum(float(q[t]) / rq * cen[ids[i]][t] for t in range(d))
+        for m in range(M):
+            acc += sum(float(q[m * dsub + t]) / rq * cb[m][codes[i][m]][t] for t in range(dsub))
+        approx.append(rq * norms[i] / math.sqrt(d) * acc)
+    k = min(n, -(-n * ppm // 1_000_000))
+    T = sorted(range(n), key=lambda i: (-approx[i], i))[:k]
+    Bset = [i for i in range(n) if i not in set(T)]
+    exact = {i: sum(float(q[t]) * K[i][t] for t in range(d)) / math.sqrt(d) for i in T}
+    count = [sum(1 for i in range(n) if ids[i] == j) for j in range(n_list)]
+    v_global = [sum(count[j] * vmeans[j][t] for j in range(n_list)) / n for t in range(d)]
+    if variant == "T" or (variant in ("C2", "C2b") and not T):
+        bg_logit = {i: -math.inf for i in Bset}
+    elif variant == "C2":
+        bg_logit = {i: sum(approx[t] for t in T) / len(T) for i in Bset}
+    elif variant == "C2b":
+        bg_logit = {i: min(exact.values()) for i in Bset}
+    else:
+        bg_logit = {i: approx[i] for i in Bset}
+    m0 = max(list(exact.values()) + list(bg_logit.values()))
+    if m0 == -math.inf:           # nothing attended (k = 0 and no background): defined as zero
+        return np.zeros(d)
+    num, den = [0.0] * d, 0.0
+    for i in T:
+        e = math.exp(exact[i] - m0)
+        den += e
+        for t in range(d):
+            num[t] += e * V[i][t]
+    for i in Bset:
+        e = math.exp(bg_logit[i] - m0)
+        if e == 0.0:
+            continue
+        j = ids[i]
+        if variant == "B":
+            val = vmeans[j]
+        elif variant == "Bx":     # mean of the list's unselected members, from the stored mean
+            t_in = [s for s in T if ids[s] == j]
+            val = [(count[j] * vmeans[j][t] - sum(V[s][t] for s in t_in)) / (count[j] - len(t_in))
+                   for t in range(d)]
+        else:
+            val = v_global
+        den += e
+        for t in range(d):
+            num[t] += e * val[t]
+    return np.array(num) / den
+
+
+@pytest.mark.parametrize("variant", ["B", "T", "Bx", "C", "C2", "C2b"])
+@pytest.mark.parametrize("seed,n,ppm", [(0, 40, 150000), (1, 23, 50000), (2, 12, 0)])
+def test_variants_against_scalar_loops(variant, seed, n, ppm):
+    rng = np.random.default_rng(100 + seed)
+    d, n_list, M, n_code = 4, 3, 2, 4
+    cen, cb, codes, ids, norms, _ = random_index(rng, n, d, n_list, M, n_code)
+    K, V, q = rng.normal(size=(n, d)), rng.normal(size=(n, d)), rng.normal(size=d)
+    vmeans = list_means(V, ids, n_list) + rng.normal(size=(n_list, d)) * 0.05   # stored, not exact
+    got = run_head(q, cen, cb, codes, ids, norms, vmeans, K, V, ppm, variant=variant)
+    want = brute_force_variant(variant, q, cen, cb, codes, ids, norms, vmeans, K, V, ppm)
+    np.testing.assert_allclose(got["y"], want, rtol=1e-10, atol=1e-12)
+
+
+def test_variant_closed_forms():
+    """Hand-checkable instances.  One list, four identical keys (all logits equal, exact codes),
+    scalar values 1, 2, 3, 4 in every dim, k = 1 (the stable rule selects position 0):
+      B   (1 + 3 * 2.5) / 4 = 2.125      the stored mean counts the selected member
+      Bx  (1 + 3 * 3.0) / 4 = 2.5        mean of the unselected members (2 + 3 + 4) / 3
+      C   one list, so the global mean is the list mean: 2.125
+      C2, C2b  shared logit = the common logit, global mean 2.5: 2.125
+      T   the selected token alone: 1"""
+    d, n = 4, 4
+    cen = np.array([[0.5, 0.0, 0.0, 0.0]])
+    cb = np.zeros((2, 4, 2))
+    codes = np.zeros((n, 2), dtype=np.uint8)
+    ids = np.zeros(n, dtype=np.int64)
+    norms = np.full(n, 2.0)
+    K = np.tile(2.0 * cen, (n, 1))
+    V = np.arange(1.0, 5.0)[:, None] * np.ones((1, d))
+    q = np.array([1.0, 0.0, 0.0, 0.0])
+    vmeans = V.mean(axis=0, keepdims=True)
+    want = dict(B=2.125, Bx=2.5, C=2.125, C2=2.125, C2b=2.125, T=1.0)
+    for variant, y in want.items():
+        r = run_head(q, cen, cb, codes, ids, norms, vmeans, K, V, 250000, variant=variant)
+        assert r["T"].tolist() == [0]
+        np.testing.assert_allclose(r["y"], np.full(d, y), rtol=1e-13)
+
+
+def test_variant_relations():
+    """T equals textbook attention over the exact set alone; Bx equals B when the values are
+    constant inside every list; C equals B when every list stores the same mean; C2b with
+    rho = 1 has no background left and is dense attention."""
+    rng = np.random.default_rng(7)
+    n, d, n_list, M, n_code = 60, 8, 4, 2, 8
+    cen, cb, codes, ids, norms, _ = random_index(rng, n, d, n_list, M, n_code)
+    K, V, q = rng.normal(size=(n, d)), rng.normal(size=(n, d)), rng.normal(size=d)
+    vmeans = list_means(V, ids, n_list)
+    t = run_head(q, cen, cb, codes, ids, norms, vmeans, K, V, 100000, n_sink=2, n_local=3, variant="T")
+    np.testing.assert_allclose(t["y"], dense_attention(q, K[t["E"]], V[t["E"]], 1 / math.sqrt(d)),
+                               rtol=1e-12)
+    assert t["Z_B"] == 0.0
+    Vc = vmeans[ids]                                          # constant inside each list
+    b = run_head(q, cen, cb, codes, ids, norms, vmeans, K, Vc, 100000, variant="B")
+    bx = run_head(q, cen, cb, codes, ids, norms, vmeans, K, Vc, 100000, variant="Bx")
+    np.testing.assert_allclose(bx["y"], b["y"], rtol=1e-10)
+    same = np.tile(rng.normal(size=(1, d)), (n_list, 1))
+    b = run_head(q, cen, cb, codes, ids, norms, same, K, V, 100000, variant="B")
+    c = run_head(q, cen, cb, codes, ids, norms, same, K, V, 100000, variant="C")
+    np.testing.assert_allclose(c["y"], b["y"], rtol=1e-12)
+    full = run_head(q, cen, cb, codes, ids, norms, vmeans, K, V, 1000000, variant="C2b")
+    np.testing.assert_allclose(full["y"], dense_attention(q, K, V, 1 / math.sqrt(d)), rtol=1e-12)

@@ -121,7 +121,7 @@ typedef enum {
   PQHSA_BUF_LUT = 0,            /* float   [B][H_kv][n_hg][256][M][Gc]                        */
   PQHSA_BUF_COARSE = 1,         /* float   [B][H_kv][n_hg][n_list][Gc]                        */
   PQHSA_BUF_SCORES = 2,         /* float   [B][H_q][N_max]                                    */
-  PQHSA_BUF_LIST_PARTIALS = 3,  /* float   [B][H_q][n_part][1 + n_list]                       */
+  PQHSA_BUF_LIST_PARTIALS = 3,  /* float   [B][H_kv][n_hg][n_part][Gc * (2 + n_list)]         */
   PQHSA_BUF_SEL_IDX = 4,        /* int32   [B][H_q][k_max]                                    */
   PQHSA_BUF_SEL_COUNT = 5,      /* int32   [B][H_q]                                           */
   PQHSA_BUF_KTH = 6             /* float   [B][H_q]                                           */
@@ -146,11 +146,13 @@ int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index
 
 /* Step 2 (Eq. 2 and the fused per-list reduction of Sec. 3.3).  seq_lens [B] int32.
  * Writes scores[b][h][i] = l~_i for the tokens i of the indexed region R_b and -inf for the
- * sink and window tokens (i < seq_lens[b]; they never compete in the top-k), and for every
- * segment s of the row (a contiguous token range scanned by one CTA; at most n_part per row,
- * the count is a function of seq_lens only) list_partials[b][h][s][0] = ref_s = max l~_i
- * over the segment's tokens of R_b (-inf if it has none) and [1+j] = sum over the segment's
- * members of list j inside R_b of exp(l~_i - ref_s). */
+ * sink and window tokens (i < seq_lens[b]; they never compete in the top-k), and the list
+ * partials: every (sequence, KV head, head group) is scanned in segments (contiguous token
+ * ranges, one per CTA; at most n_part, the count is a function of seq_lens only), and segment s
+ * leaves list_partials[b][kv][hg][s] = { ref[Gc], max[Gc], sum[n_list][Gc] } with, for head g of
+ * the group, max[g] = max l~_i over the segment's tokens of R_b (-inf if it has none), ref[g] =
+ * the reference of the sums (any value the segment chose; -inf if it has no token of R_b) and
+ * sum[j][g] = sum over the segment's members of list j inside R_b of exp(l~_i - ref[g]). */
 int pqhsa_scan(const pqhsa_params* params, const pqhsa_index* index, const float* lut,
                const float* coarse, const int32_t* seq_lens, float* scores,
                float* list_partials, void* ws, size_t ws_bytes, void* stream);

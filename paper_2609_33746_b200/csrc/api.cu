@@ -3,7 +3,6 @@
 // except pqhsa_last_device_status and pqhsa_decode_host, which say so.
 #include <mutex>
 
-#include <cstdlib>
 #include "common.cuh"
 
 namespace pqhsa {
@@ -85,12 +84,12 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (o.n_part > kMaxSeg) return PQHSA_ERR_UNSUPPORTED;     // more SMs than this build plans for
   o.rows = o.B * o.Hq;
   // the coarse table is bulk-copied: its byte size and unit stride must be multiples of 16.
-  // Prefer a 3-stage code ring with the coarse table in shared memory, then give up the
-  // coarse table, then a stage.
+  // Prefer the coarse table in shared memory (a random 16-byte read per token either way, but
+  // without a tag lookup), then a third stage of the code ring.
   const bool co_ok = (o.Gc * o.n_list) % 4 == 0;
   if (co_ok && scan_smem_bytes(o, true, 3) <= kMaxSmemPerCta) { o.coarse_in_smem = 1; o.scan_stages = 3; }
-  else if (scan_smem_bytes(o, false, 3) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 3; }
   else if (co_ok && scan_smem_bytes(o, true, 2) <= kMaxSmemPerCta) { o.coarse_in_smem = 1; o.scan_stages = 2; }
+  else if (scan_smem_bytes(o, false, 3) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 3; }
   else if (scan_smem_bytes(o, false, 2) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 2; }
   else return PQHSA_ERR_UNSUPPORTED;
 
@@ -126,12 +125,6 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (o.bg_ctas > 8) o.bg_ctas = 8;
   if (o.bg_ctas < ceil_div(o.k_max, 768)) o.bg_ctas = ceil_div(o.k_max, 768);   // 6 tokens per thread
   if (o.bg_ctas < 1) o.bg_ctas = 1;
-#ifdef PQHSA_TUNE
-  if (const char* e = getenv("PQHSA_HIST_CHUNKS")) o.hist_chunks = atoi(e);
-  if (const char* e = getenv("PQHSA_SPLITS")) o.splits = atoi(e);
-  if (const char* e = getenv("PQHSA_BG_CTAS")) o.bg_ctas = atoi(e);
-  if (const char* e = getenv("PQHSA_BG_SPLITS")) o.bg_splits = atoi(e);
-#endif
   return PQHSA_OK;
 }
 
@@ -141,7 +134,7 @@ static size_t buffer_elems(const Plan& pl, int which) {
     case PQHSA_BUF_LUT: return units * pl.n_code * pl.M * pl.Gc;
     case PQHSA_BUF_COARSE: return units * pl.n_list * pl.Gc;
     case PQHSA_BUF_SCORES: return (size_t)pl.rows * pl.N_max;
-    case PQHSA_BUF_LIST_PARTIALS: return (size_t)pl.rows * pl.n_part * (pl.n_list + 1);
+    case PQHSA_BUF_LIST_PARTIALS: return units * pl.n_part * pl.Gc * (pl.n_list + 2);
     case PQHSA_BUF_SEL_IDX: return (size_t)pl.rows * pl.k_max;
     case PQHSA_BUF_SEL_COUNT: return (size_t)pl.rows;
     case PQHSA_BUF_KTH: return (size_t)pl.rows;

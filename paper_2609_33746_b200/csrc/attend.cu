@@ -70,12 +70,18 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   const long long s_u = base + (long long)(kv * pl.n_hg + hg) * tb;
   const int c_first = split_cta_of(sp, s_u);
   const int nseg = min(kMaxSeg, split_cta_of(sp, s_u + tb - 1) - c_first + 1);
-  const float* pr = partials + (size_t)row * pl.n_part * (n_list + 1);
+  // the unit's partials: per segment a header [2 Gc] (reference, maximum per head) and the sums
+  // [n_list][Gc] relative to the reference
+  const int Gc = pl.Gc, g = (h % pl.G) % Gc;
+  const size_t seg_stride = (size_t)Gc * (n_list + 2);
+  const float* pr = partials + (((size_t)b * pl.Hkv + kv) * pl.n_hg + hg) * pl.n_part * seg_stride;
 
-  for (int sg = tid; sg < nseg; sg += kBgThreads)                      // segment maxima
-    s_scale[sg] = pr[(size_t)sg * (n_list + 1)];
-  __syncthreads();
   float m = -CUDART_INF_F;
+  for (int sg = tid; sg < nseg; sg += kBgThreads) {                    // segment maxima
+    const float v = pr[(size_t)sg * seg_stride + Gc + g];
+    s_scale[sg] = v;
+  }
+  __syncthreads();
   for (int s = 0; s < nseg; ++s) m = fmaxf(m, s_scale[s]);
   if (!(m > -CUDART_INF_F)) {            // no token of R in this row: no background at all
     if (c == 0 && tid == 0) bg_max[row] = -CUDART_INF_F;
@@ -83,17 +89,21 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   }
   const float m2 = m * kLog2e;
   __syncthreads();
-  for (int sg = tid; sg < nseg; sg += kBgThreads)
-    s_scale[sg] = fast_exp2(fmaf(s_scale[sg], kLog2e, -m2));
+  for (int sg = tid; sg < nseg; sg += kBgThreads) {
+    // a segment's sums are relative to its reference: exp2(l~ log2 e - ref log2 e)
+    const float ref = pr[(size_t)sg * seg_stride + g];
+    s_scale[sg] = s_scale[sg] > -CUDART_INF_F ? fast_exp2(ref * kLog2e - m2) : 0.f;
+  }
   __syncthreads();
   const int jl = (int)((long long)c * n_list / C), jh = (int)((long long)(c + 1) * n_list / C);
+  const float* sums = pr + 2 * Gc + g;
   for (int j = jl + tid; j < jh; j += kBgThreads) {
     float acc = 0.f;
     for (int s0 = 0; s0 < nseg; s0 += 8) {
       float v[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u)
-        v[u] = (s0 + u < nseg) ? pr[(size_t)(s0 + u) * (n_list + 1) + 1 + j] : 0.f;
+        v[u] = (s0 + u < nseg) ? sums[(size_t)(s0 + u) * seg_stride + (size_t)j * Gc] : 0.f;
 #pragma unroll
       for (int u = 0; u < 8; ++u)
         if (s0 + u < nseg) acc = fmaf(v[u], s_scale[s0 + u], acc);

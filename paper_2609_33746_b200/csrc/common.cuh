@@ -14,10 +14,7 @@ namespace pqhsa {
 constexpr int kHeadDim = 128;
 constexpr int kNCode = 256;
 constexpr int kTile = 32;            // tokens per scan tile: one token per lane
-#ifndef PQHSA_SCAN_THREADS
-#define PQHSA_SCAN_THREADS 512
-#endif
-constexpr int kScanThreads = PQHSA_SCAN_THREADS;
+constexpr int kScanThreads = 512;
 constexpr int kScanMinTiles = kScanThreads / 32;   // a scan CTA gets at least one tile per warp
 constexpr int kMaxSeg = 320;                       // scan segments one unit may be cut into (n_part)
 constexpr int kHistBins = 4096;      // 12-bit radix digits of the select's shared-memory histograms
@@ -50,7 +47,7 @@ struct Plan {
   int bg_splits;                     // background CTAs per (sequence, KV head, head group) there
   int bg_ctas;                       // CTAs per row in the background preparation
   int coarse_in_smem;                // scan keeps the coarse table in shared memory
-  int scan_stages;                   // cp.async stages per warp in the scan's code ring (3 or 2)
+  int scan_stages;                   // stages per warp in the scan's code ring (3 or 2)
   int num_sms;
 };
 

@@ -10,18 +10,26 @@
 // positions static each lane permutes its own code bytes once per token
 // (byte p <- byte p ^ (lane & 7)).
 //
-// The codes stream from HBM through a per-warp ring of cp.async stages in shared memory
-// (kStages tiles of 32 tokens in flight per warp), so the bytes in flight do not depend on
-// registers; 16-byte chunks are placed with an XOR swizzle that makes the lane-per-token
-// 16-byte reads conflict free as well.  Norms and list ids (6 bytes per token) are
-// prefetched one tile ahead in registers.
+// The table reads bound the kernel: 16 bytes of shared memory per token, subspace and head
+// group against 128 bytes per SM and clock, and the same load/store data pipe also carries
+// every other shared or global access of the SM (measured: the kernel runs at one wavefront
+// of that pipe per clock).  So everything else is kept as light on that pipe as it can be:
+//   * the codes stream from HBM through a per-warp ring of cp.async stages in shared memory
+//     (kStages tiles of 32 tokens in flight per warp), so the bytes in flight do not depend on
+//     registers; 16-byte chunks are placed with an XOR swizzle that makes the lane-per-token
+//     16-byte reads conflict free as well.  Norms and list ids (6 bytes per token) are
+//     prefetched one tile ahead in registers;
+//   * the per-list exp-sums are not kept in shared memory, where a float atomic is a
+//     compare-and-swap loop: the CTA's partial for its segment lives in global memory
+//     ([list][head], L2 resident) and every token adds its Gc terms with ONE fire-and-forget
+//     vector reduction (red.global.add.v4.f32), resolved in L2.
 //
 // Per-list exp-sums: the CTA takes the maximum logit of its first round of tiles (one tile
-// per warp) as reference and adds exp(l~ - ref) into a [Gc][n_list] table in shared memory
-// while it scans.  When the segment is done the sums are re-based to the segment's true
-// maximum and flushed as one partial (maximum + sums) per (score row, CTA segment).  If some
-// logit exceeds the reference by so much that exp could overflow, the CTA discards the table
-// and rebuilds it in a second pass over the scores it has just written (L2 hits).
+// per warp) as reference ref_s and adds exp(l~ - ref_s) for every token of R.  The partial's
+// header keeps ref_s and the segment's true maximum; the consumer (background preparation)
+// re-bases the segments of a unit to the row's maximum.  If some logit exceeds the reference
+// by so much that exp could overflow, the CTA clears its partial and rebuilds it against the
+// true maximum in a second pass over the scores it has just written (L2 hits).
 #include "common.cuh"
 
 namespace pqhsa {
@@ -76,6 +84,16 @@ template <> __device__ __forceinline__ void load_vec<2>(float (&f)[2], const flo
 template <> __device__ __forceinline__ void load_vec<4>(float (&f)[4], const float* p) {
   const float4 v = *reinterpret_cast<const float4*>(p);
   f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+
+template <int GC> __device__ __forceinline__ void red_add(float* dst, const float (&e)[GC]) {
+  if constexpr (GC == 4)
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(e[0]), "f"(e[1]),
+                 "f"(e[2]), "f"(e[3]) : "memory");
+  else if constexpr (GC == 2)
+    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dst), "f"(e[0]), "f"(e[1]) : "memory");
+  else
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(e[0]) : "memory");
 }
 
 constexpr float kOverflowGuardLog2 = 96.0f;   // exp2 arguments above this trigger the rebuild
@@ -207,18 +225,14 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   constexpr int kEntryBytes = GC * 4;
   constexpr int kRowBytes = M * kEntryBytes;       // stride between consecutive z
   constexpr int kWarps = kScanThreads / 32;
-#ifndef PQHSA_SCAN_BLK
-#define PQHSA_SCAN_BLK 8
-#endif
-  constexpr int kBlk = PQHSA_SCAN_BLK;             // table reads issued back to back
+  constexpr int kBlk = 8;             // table reads issued back to back
 
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* s_lut = reinterpret_cast<float*>(smem_raw);
-  float* s_sums = s_lut + kLutFloats;                       // [GC][n_list]
-  float* s_coarse = s_sums + GC * pl.n_list;                // [n_list][GC] when it fits
+  float* s_coarse = s_lut + kLutFloats;                     // [n_list][GC] when it fits
   // the code ring sits behind the tables: kStages tiles per warp
   const uint32_t table_bytes =
-      uint32_t(kLutFloats + GC * pl.n_list * (pl.coarse_in_smem ? 2 : 1)) * 4u;
+      uint32_t(kLutFloats + (pl.coarse_in_smem ? GC * pl.n_list : 0)) * 4u;
   const uint32_t ring0 = smem_u32(smem_raw) + ((table_bytes + 127u) & ~127u) +
                          uint32_t((threadIdx.x >> 5) * kStages * CodeTile<kCB>::kBytes);
   __shared__ float s_red[kWarps][GC];
@@ -251,6 +265,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   const int lx = lane & 7;
   const uint32_t byte_sel = 0x3210u ^ (uint32_t(lane & 3) * 0x1111u);
   const bool swap_words = (lane & 4) != 0;
+  const uint32_t byte_sel2 = byte_sel + (swap_words ? 0x4444u : 0u);
   uint32_t lane_off[8];   // shared-window address of entry (z = 0, m = t ^ lx) for t = s & 7
 #pragma unroll
   for (int t = 0; t < 8; ++t) lane_off[t] = smem_u32(s_lut) + uint32_t((t ^ lx) * kEntryBytes);
@@ -281,6 +296,9 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     const int n_heads = min(GC, pl.G - hg * GC);             // real heads in this head group
     const float* g_coarse = coarse + unit * (size_t)n_list * GC;
     const int tend = t0 + cnt;
+    // this CTA's partial of the unit: header [2 GC] (reference, maximum), sums [n_list][GC]
+    float* part = partials + (unit * pl.n_part + slot) * (size_t)(GC * (n_list + 2));
+    float* part_sums = part + 2 * GC;
 
     __syncthreads();   // previous segment's tables are no longer in use
     if (tid == 0) {
@@ -291,7 +309,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
       if (co_bytes) bulk_g2s(s_coarse, g_coarse, co_bytes, &s_bar);
       s_overflow = 0;
     }
-    for (int i = tid; i < GC * n_list; i += kScanThreads) s_sums[i] = 0.f;
+    for (int i = tid; i < GC * n_list; i += kScanThreads) part_sums[i] = 0.f;
 
     // prologue of the ring: the first kStages-1 tiles of this warp (overlaps the table copy)
     int t = t0 + warp;
@@ -303,7 +321,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     load_meta(cur, lids, norms, row_base, t * kTile + lane, t < tend && t * kTile + lane < Nb);
     if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, 4);
     bar_parity ^= 1u;
-    __syncthreads();   // s_sums zeroed, tables landed
+    __syncthreads();   // partial zeroed, tables landed
 
     float mx[GC], ref2[GC];
 #pragma unroll
@@ -359,8 +377,8 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
 #pragma unroll
         for (int j = 0; j < M / 8; ++j) {
           const uint32_t a = raw[2 * j], bb = raw[2 * j + 1];
-          cw[2 * j] = __byte_perm(swap_words ? bb : a, 0u, byte_sel);
-          cw[2 * j + 1] = __byte_perm(swap_words ? a : bb, 0u, byte_sel);
+          cw[2 * j] = __byte_perm(a, bb, byte_sel2);
+          cw[2 * j + 1] = __byte_perm(a, bb, byte_sel2 ^ 0x4444u);
         }
 #pragma unroll
         for (int sb = 0; sb < M; sb += kBlk) {
@@ -381,8 +399,9 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         acc0.merge(acc1);
         float accf[GC], co[GC];
         acc0.get(accf);
-        if (pl.coarse_in_smem) load_vec<GC>(co, s_coarse + cur.lid * GC);
-        else load_vec<GC>(co, g_coarse + cur.lid * GC);
+        // (a list id outside [0, n_list) is an index error, not a reason to read out of bounds)
+        if (pl.coarse_in_smem) load_vec<GC>(co, s_coarse + min(cur.lid, (uint32_t)(n_list - 1)) * GC);
+        else load_vec<GC>(co, g_coarse + min(cur.lid, (uint32_t)(n_list - 1)) * GC);
         if (valid) {
           // sink and window tokens are attended exactly: their score is -inf, so that the
           // top-k never picks them and they add nothing to the list sums
@@ -412,26 +431,25 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
 #pragma unroll
           for (int ww = 0; ww < kWarps; ++ww) v = fmaxf(v, s_red[ww][g]);
           ref2[g] = v * kLog2e;
+          if (tid == g) s_ref[g] = v;                    // header value: same units as the scores
         }
-        if (tid < GC) s_ref[tid] = ref2[tid];
         first = false;
       }
-      if (in_r) {
+      {
+        // a token outside R has score -inf and adds exp2(-inf) = 0 (or, against a reference of
+        // -inf, a NaN that no comparison below accepts)
         float x[GC], xm = -CUDART_INF_F;
 #pragma unroll
         for (int g = 0; g < GC; ++g) {
-          x[g] = fmaf(sc[g], kLog2e, -ref2[g]);      // -inf for padded head slots
+          x[g] = fmaf(sc[g], kLog2e, -ref2[g]);
           xm = fmaxf(xm, x[g]);
         }
+        if (xm > kOverflowGuardLog2) s_overflow = 1;
         if (xm > kNegligibleLog2) {
-          if (xm > kOverflowGuardLog2) {
-            s_overflow = 1;
-          } else {
+          float e[GC];
 #pragma unroll
-            for (int g = 0; g < GC; ++g)
-              if (x[g] > kNegligibleLog2)
-                atomicAdd(&s_sums[g * n_list + cur.lid], fast_exp2(x[g]));
-          }
+          for (int g = 0; g < GC; ++g) e[g] = fast_exp2(x[g]);
+          red_add<GC>(part_sums + min(cur.lid, (uint32_t)(n_list - 1)) * GC, e);
         }
       }
       cur = nxt;
@@ -457,33 +475,39 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     __syncthreads();   // also orders this CTA's score stores before the rebuild's loads
 
     if (s_overflow) {
-      // rare: rebuild the table against the true maximum from the scores just written
-      for (int i = tid; i < GC * n_list; i += kScanThreads) s_sums[i] = 0.f;
+      // rare: rebuild the partial against the true maximum from the scores just written.
+      // The reductions in flight target the same addresses as the clearing stores, so they
+      // are fenced first.
+      __threadfence();
       __syncthreads();
-      if (tid < GC) s_ref[tid] = s_max[tid] * kLog2e;
+      for (int i = tid; i < GC * n_list; i += kScanThreads) part_sums[i] = 0.f;
+      if (tid < GC) s_ref[tid] = s_max[tid];
+      __threadfence();
       __syncthreads();
       const int i_begin = t0 * kTile;
       const int i_end = min(Nb, tend * kTile);
       for (int i = i_begin + tid; i < i_end; i += kScanThreads) {
-        const uint32_t lid = __ldg(lids + row_base + i);
+        const uint32_t lid = min((uint32_t)__ldg(lids + row_base + i), (uint32_t)(n_list - 1));
+        float e[GC];
+        bool any = false;
 #pragma unroll
         for (int g = 0; g < GC; ++g) {
+          e[g] = 0.f;
           if (g < n_heads) {
             const float s = __ldcg(scores + (size_t)(row0 + g) * N_max + i);
-            const float x = fmaf(s, kLog2e, -s_ref[g]);     // -inf or NaN outside R
-            if (x > kNegligibleLog2) atomicAdd(&s_sums[g * n_list + lid], fast_exp2(x));
+            const float x = fmaf(s, kLog2e, -(s_ref[g] * kLog2e));     // -inf outside R
+            if (x > kNegligibleLog2) { e[g] = fast_exp2(x); any = true; }
           }
         }
+        if (any) red_add<GC>(part_sums + (size_t)lid * GC, e);
       }
-      __syncthreads();
     }
-    // flush: header = segment maximum, sums re-based from the reference to that maximum
-    for (int idx = tid; idx < n_heads * (n_list + 1); idx += kScanThreads) {
-      const int g = idx / (n_list + 1), j = idx - g * (n_list + 1);
-      // a segment without any token of R has maximum -inf and empty sums
-      const float rescale = s_max[g] > -CUDART_INF_F ? fast_exp2(s_ref[g] - s_max[g] * kLog2e) : 0.f;
-      const float v = (j == 0) ? s_max[g] : s_sums[g * n_list + j - 1] * rescale;
-      partials[((size_t)(row0 + g) * pl.n_part + slot) * (n_list + 1) + j] = v;
+    // header: the reference the sums are relative to (same units as the scores; the exponent
+    // was formed as fma(l~, log2 e, -(ref * log2 e)) in base 2) and the segment's maximum; a
+    // segment without any token of R has both at -inf
+    if (tid < GC) {
+      part[tid] = s_max[tid] > -CUDART_INF_F ? s_ref[tid] : -CUDART_INF_F;
+      part[GC + tid] = s_max[tid];
     }
 
     lo += cnt;
@@ -496,7 +520,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
 }
 
 size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem, int stages) {
-  size_t f = (size_t)pl.n_code * pl.M * pl.Gc + (size_t)pl.Gc * pl.n_list;
+  size_t f = (size_t)pl.n_code * pl.M * pl.Gc;
   if (coarse_in_smem) f += (size_t)pl.Gc * pl.n_list;
   const size_t tables = (f * sizeof(float) + 127) / 128 * 128;    // the ring is 128-byte aligned
   return tables + (size_t)(kScanThreads / 32) * stages * kTile * pl.code_bytes;

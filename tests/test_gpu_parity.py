@@ -161,8 +161,12 @@ def test_stage_scan_scores_and_list_sums(key):
     torch.cuda.synchronize()
     n_part = pqhsa.num_partials(op.params)
     N_max = op.params.max_seq_len
+    Gc = pqhsa.heads_per_group(op.params)
+    n_hg = (cfg.group + Gc - 1) // Gc
     scores = op.scores.view(cfg.batch, cfg.n_q_heads, N_max).cpu().double().numpy()
-    parts = op.list_partials.view(cfg.batch, cfg.n_q_heads, n_part, cfg.n_list + 1).cpu().double().numpy()
+    # per (sequence, KV head, head group, segment): ref[Gc], max[Gc], sums[n_list][Gc]
+    parts = op.list_partials.view(cfg.batch, cfg.n_kv_heads, n_hg, n_part,
+                                  cfg.n_list + 2, Gc).cpu().double().numpy()
     for (b, h), r in ref.items():
         n = int(arrays["seq_lens"][b])
         R = r["R"]                                      # indexed region: positions r0 .. r1-1
@@ -176,12 +180,15 @@ def test_stage_scan_scores_and_list_sums(key):
         if len(R) == 0:
             continue
         # per-list exp-sums over ALL members, merged over the scan's segments
-        p = parts[b, h]
-        used = ~np.isnan(p[:, 0])
+        kv, hh = divmod(h, cfg.group)
+        hg, g = divmod(hh, Gc)
+        p = parts[b, kv, hg]                            # [n_part][2 + n_list][Gc]
+        p_ref, p_max, p_sum = p[:, 0, g], p[:, 1, g], p[:, 2:, g]
+        used = ~np.isnan(p_max) & ~np.isneginf(p_max)
         assert used.any()
-        m = p[used, 0].max()
+        m = p_max[used].max()
         assert abs(m - want.max()) <= LOGIT_RTOL * max(1.0, abs(want.max()))
-        tot = (p[used, 1:] * np.exp(p[used, 0] - m)[:, None]).sum(axis=0)
+        tot = (p_sum[used] * np.exp(p_ref[used] - m)[:, None]).sum(axis=0)
         lists = arrays["list_ids"][b, h // cfg.group, r0:r1].astype(np.int64)
         want_tot = np.bincount(lists, weights=np.exp(want - want.max()), minlength=cfg.n_list)
         assert np.abs(tot - want_tot).max() <= 2e-4 * want_tot.sum()

@@ -50,7 +50,7 @@ def test_size_arithmetic_for_the_128k_workload():
     assert pqhsa.buffer_elems(p, pqhsa.BUF_LUT) == 8 * 256 * 32 * 4
     assert pqhsa.buffer_elems(p, pqhsa.BUF_COARSE) == 8 * 1024 * 4
     assert pqhsa.buffer_elems(p, pqhsa.BUF_SCORES) == 32 * 131072
-    assert pqhsa.buffer_elems(p, pqhsa.BUF_LIST_PARTIALS) == 32 * n_part * 1025
+    assert pqhsa.buffer_elems(p, pqhsa.BUF_LIST_PARTIALS) == 8 * n_part * 4 * (1024 + 2)
     assert pqhsa.buffer_elems(p, pqhsa.BUF_SEL_IDX) == 32 * 1311
     ws = pqhsa.workspace_bytes(p)
     assert ws > 4 * 32 * 131072 and ws % 256 == 0

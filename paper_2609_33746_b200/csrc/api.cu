@@ -77,8 +77,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.k_max = p->k_max; o.n_sink = p->n_sink; o.n_local = p->n_local;
   o.exact_multiple = p->exact_set_multiple; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
   o.num_sms = sm_count();
-  // persistent scan CTAs: one per SM, two with the small tables of 4-bit codes
-  o.scan_ctas = o.n_code == 16 ? 2 * o.num_sms : o.num_sms;
+  o.scan_ctas = o.num_sms;                                  // persistent scan CTAs: one per SM
   o.upb = o.Hkv * o.n_hg;
   o.n_part = o.scan_ctas / o.upb + 2;
   if (o.n_part > kMaxSeg) return PQHSA_ERR_UNSUPPORTED;     // more SMs than this build plans for
@@ -87,6 +86,14 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   // Prefer the coarse table in shared memory (a random 16-byte read per token either way, but
   // without a tag lookup), then a third stage of the code ring.
   const bool co_ok = (o.Gc * o.n_list) % 4 == 0;
+  if (o.n_code == 16) {
+    // 4-bit scan: the table is tiny, so the coarse table gets a conflict-free 128-byte row per
+    // list when that fits, else one entry per list, else it stays in global memory
+    o.scan_stages = 0;
+    if (scan4_smem_bytes(o, 2) <= kMaxSmemPerCta) o.coarse_in_smem = 2;
+    else if (co_ok && scan4_smem_bytes(o, 1) <= kMaxSmemPerCta) o.coarse_in_smem = 1;
+    else o.coarse_in_smem = 0;
+  } else
   if (co_ok && scan_smem_bytes(o, true, 3) <= kMaxSmemPerCta) { o.coarse_in_smem = 1; o.scan_stages = 3; }
   else if (co_ok && scan_smem_bytes(o, true, 2) <= kMaxSmemPerCta) { o.coarse_in_smem = 1; o.scan_stages = 2; }
   else if (scan_smem_bytes(o, false, 3) <= kMaxSmemPerCta) { o.coarse_in_smem = 0; o.scan_stages = 3; }

@@ -46,7 +46,8 @@ struct Plan {
   int splits;                        // exact (split-K) CTAs per row in the attend kernel
   int bg_splits;                     // background CTAs per (sequence, KV head, head group) there
   int bg_ctas;                       // CTAs per row in the background preparation
-  int coarse_in_smem;                // scan keeps the coarse table in shared memory
+  int coarse_in_smem;                // scan keeps the coarse table in shared memory (4-bit scan: 2 =
+                                     // one conflict-free 128-byte row per list)
   int scan_stages;                   // stages per warp in the scan's code ring (3 or 2)
   int num_sms;
 };
@@ -227,6 +228,10 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
                           const float* list_partials, const int32_t* sel_idx,
                           const int32_t* sel_count, const int32_t* seq_lens, void* out,
                           float* lse, cudaStream_t st);
+cudaError_t launch_scan4(const Plan& pl, const pqhsa_index& ix, const float* lut,
+                         const float* coarse, const int32_t* seq_lens, float* scores,
+                         float* list_partials, int* status, cudaStream_t st);
 size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem, int stages);
+size_t scan4_smem_bytes(const Plan& pl, int coarse_mode);
 
 }  // namespace pqhsa

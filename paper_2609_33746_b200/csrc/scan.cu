@@ -30,74 +30,9 @@
 // re-bases the segments of a unit to the row's maximum.  If some logit exceeds the reference
 // by so much that exp could overflow, the CTA clears its partial and rebuilds it against the
 // true maximum in a second pass over the scores it has just written (L2 hits).
-#include "common.cuh"
+#include "scan_common.cuh"
 
 namespace pqhsa {
-
-// Packed accumulators: the Gc partial sums of a token live in 64-bit registers holding two
-// floats each, so one table entry is added with add.f32x2 (two lanes per instruction).
-template <int GC> struct Acc;
-template <> struct Acc<4> {
-  unsigned long long lo, hi;
-  __device__ __forceinline__ void zero() { lo = 0ull; hi = 0ull; }
-  __device__ __forceinline__ void load(uint32_t saddr) {
-    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(lo), "=l"(hi) : "r"(saddr));
-  }
-  __device__ __forceinline__ void merge(const Acc& o) {
-    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(lo) : "l"(o.lo));
-    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(hi) : "l"(o.hi));
-  }
-  __device__ __forceinline__ void get(float (&f)[4]) const {
-    f[0] = __uint_as_float((uint32_t)lo); f[1] = __uint_as_float((uint32_t)(lo >> 32));
-    f[2] = __uint_as_float((uint32_t)hi); f[3] = __uint_as_float((uint32_t)(hi >> 32));
-  }
-};
-template <> struct Acc<2> {
-  unsigned long long lo;
-  __device__ __forceinline__ void zero() { lo = 0ull; }
-  __device__ __forceinline__ void load(uint32_t saddr) {
-    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(lo) : "r"(saddr));
-  }
-  __device__ __forceinline__ void merge(const Acc& o) {
-    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(lo) : "l"(o.lo));
-  }
-  __device__ __forceinline__ void get(float (&f)[2]) const {
-    f[0] = __uint_as_float((uint32_t)lo); f[1] = __uint_as_float((uint32_t)(lo >> 32));
-  }
-};
-template <> struct Acc<1> {
-  float v;
-  __device__ __forceinline__ void zero() { v = 0.f; }
-  __device__ __forceinline__ void load(uint32_t saddr) {
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(saddr));
-  }
-  __device__ __forceinline__ void merge(const Acc& o) { v += o.v; }
-  __device__ __forceinline__ void get(float (&f)[1]) const { f[0] = v; }
-};
-
-template <int GC> __device__ __forceinline__ void load_vec(float (&f)[GC], const float* p);
-template <> __device__ __forceinline__ void load_vec<1>(float (&f)[1], const float* p) { f[0] = *p; }
-template <> __device__ __forceinline__ void load_vec<2>(float (&f)[2], const float* p) {
-  const float2 v = *reinterpret_cast<const float2*>(p);
-  f[0] = v.x; f[1] = v.y;
-}
-template <> __device__ __forceinline__ void load_vec<4>(float (&f)[4], const float* p) {
-  const float4 v = *reinterpret_cast<const float4*>(p);
-  f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
-}
-
-template <int GC> __device__ __forceinline__ void red_add(float* dst, const float (&e)[GC]) {
-  if constexpr (GC == 4)
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(e[0]), "f"(e[1]),
-                 "f"(e[2]), "f"(e[3]) : "memory");
-  else if constexpr (GC == 2)
-    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dst), "f"(e[0]), "f"(e[1]) : "memory");
-  else
-    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst), "f"(e[0]) : "memory");
-}
-
-constexpr float kOverflowGuardLog2 = 96.0f;   // exp2 arguments above this trigger the rebuild
-constexpr int kMbarSpinLimit = 1 << 22;
 
 struct TokenMeta {
   float norm;          // r_i
@@ -181,46 +116,15 @@ __device__ __forceinline__ void read_codes(uint32_t slot, int lane, uint32_t (&w
   }
 }
 
-// ---- bulk async copy global -> shared, completion on an mbarrier (TMA, no tensor map)
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
-               "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-// Bounded wait: returns false if the phase did not complete within the spin limit.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (int it = 0; it < kMbarSpinLimit; ++it) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    if (done) return true;
-  }
-  return false;
-}
-
-// kBits = 8: one byte per code, 256-entry tables.  kBits = 4: two codes per byte (subspace 2j in
-// the low nibble of byte j), 16-entry tables.
-template <int M, int GC, int kStages, int kBits>
-__global__ void __launch_bounds__(kScanThreads, kBits == 4 ? 2 : 1)
+// One byte per code, 256-entry tables (4-bit codes: scan4.cu).
+template <int M, int GC, int kStages>
+__global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restrict__ lids,
             const float* __restrict__ norms, const float* __restrict__ lut,
             const float* __restrict__ coarse, const int32_t* __restrict__ seq_lens,
             float* __restrict__ scores, float* __restrict__ partials, int* __restrict__ status) {
-  constexpr int kCodes = kBits == 4 ? 16 : 256;       // codewords per subspace
-  constexpr int kCB = kBits == 4 ? M / 2 : M;         // bytes of codes per token
+  constexpr int kCodes = 256;                         // codewords per subspace
+  constexpr int kCB = M;                              // bytes of codes per token
   constexpr int kLutFloats = kCodes * M * GC;
   constexpr int kEntryBytes = GC * 4;
   constexpr int kRowBytes = M * kEntryBytes;       // stride between consecutive z
@@ -350,27 +254,6 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         Acc<GC> acc0, acc1;
         acc0.zero();
         acc1.zero();
-        if constexpr (kBits == 4) {
-          // nibble m of the lane's code word(s); at step s the lane looks up m = s ^ (lane & 7)
-          // inside its group of 8 subspaces, as in the 8-bit path
-          uint32_t cw4[kCB / 4];
-          read_codes<kCB>(ring0 + (it % kStages) * CodeTile<kCB>::kBytes, lane, cw4);
-#pragma unroll
-          for (int sb = 0; sb < M; sb += kBlk) {
-            Acc<GC> v[kBlk];
-#pragma unroll
-            for (int u = 0; u < kBlk; ++u) {
-              const int s = sb + u;
-              const uint32_t z = (cw4[s >> 3] >> (4 * ((s & 7) ^ lx))) & 15u;
-              v[u].load(lane_off[s & 7] + z * uint32_t(kRowBytes) + uint32_t((s & ~7) * kEntryBytes));
-            }
-#pragma unroll
-            for (int u = 0; u < kBlk; u += 2) {
-              acc0.merge(v[u]);
-              acc1.merge(v[u + 1]);
-            }
-          }
-        } else {
         // position p of the lane's code array <- original byte p ^ (lane & 7)
         uint32_t raw[M / 4], cw[M / 4];
         read_codes<M>(ring0 + (it % kStages) * CodeTile<M>::kBytes, lane, raw);
@@ -394,7 +277,6 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
             acc0.merge(v[u]);
             acc1.merge(v[u + 1]);
           }
-        }
         }
         acc0.merge(acc1);
         float accf[GC], co[GC];
@@ -526,15 +408,15 @@ size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem, int stages) {
   return tables + (size_t)(kScanThreads / 32) * stages * kTile * pl.code_bytes;
 }
 
-template <int M, int GC, int S, int kBits>
+template <int M, int GC, int S>
 static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const float* lut,
                                  const float* coarse, const int32_t* seq_lens, float* scores,
                                  float* partials, int* status, cudaStream_t st) {
   const size_t smem = scan_smem_bytes(pl, pl.coarse_in_smem != 0, S);
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S, kBits>,
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(scan_kernel<M, GC, S, kBits>, dim3(pl.scan_ctas), dim3(kScanThreads), smem, st, pl,
+  return launch_pdl(scan_kernel<M, GC, S>, dim3(pl.scan_ctas), dim3(kScanThreads), smem, st, pl,
                     ix.codes, ix.list_ids, ix.key_norms, lut, coarse, seq_lens, scores, partials,
                     status);
 }
@@ -542,20 +424,20 @@ static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const fl
 cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,
                         const float* coarse, const int32_t* seq_lens, float* scores,
                         float* list_partials, int* status, cudaStream_t st) {
-#define PQHSA_SCAN_CASE(MM, GG, BITS)                                                         \
-  if (pl.M == MM && pl.Gc == GG && pl.n_code == (BITS == 4 ? 16 : 256)) {                     \
+  if (pl.n_code == 16)
+    return launch_scan4(pl, ix, lut, coarse, seq_lens, scores, list_partials, status, st);
+#define PQHSA_SCAN_CASE(MM, GG)                                                               \
+  if (pl.M == MM && pl.Gc == GG) {                                                            \
     if (pl.scan_stages >= 3)                                                                  \
-      return launch_scan_t<MM, GG, 3, BITS>(pl, ix, lut, coarse, seq_lens, scores,            \
-                                            list_partials, status, st);                       \
-    return launch_scan_t<MM, GG, 2, BITS>(pl, ix, lut, coarse, seq_lens, scores,              \
-                                          list_partials, status, st);                         \
+      return launch_scan_t<MM, GG, 3>(pl, ix, lut, coarse, seq_lens, scores, list_partials,   \
+                                      status, st);                                            \
+    return launch_scan_t<MM, GG, 2>(pl, ix, lut, coarse, seq_lens, scores, list_partials,     \
+                                    status, st);                                              \
   }
-  PQHSA_SCAN_CASE(8, 1, 8) PQHSA_SCAN_CASE(8, 2, 8) PQHSA_SCAN_CASE(8, 4, 8)
-  PQHSA_SCAN_CASE(16, 1, 8) PQHSA_SCAN_CASE(16, 2, 8) PQHSA_SCAN_CASE(16, 4, 8)
-  PQHSA_SCAN_CASE(32, 1, 8) PQHSA_SCAN_CASE(32, 2, 8) PQHSA_SCAN_CASE(32, 4, 8)
-  PQHSA_SCAN_CASE(64, 1, 8) PQHSA_SCAN_CASE(64, 2, 8)
-  PQHSA_SCAN_CASE(8, 1, 4) PQHSA_SCAN_CASE(8, 2, 4) PQHSA_SCAN_CASE(8, 4, 4)
-  PQHSA_SCAN_CASE(16, 1, 4) PQHSA_SCAN_CASE(16, 2, 4) PQHSA_SCAN_CASE(16, 4, 4)
+  PQHSA_SCAN_CASE(8, 1) PQHSA_SCAN_CASE(8, 2) PQHSA_SCAN_CASE(8, 4)
+  PQHSA_SCAN_CASE(16, 1) PQHSA_SCAN_CASE(16, 2) PQHSA_SCAN_CASE(16, 4)
+  PQHSA_SCAN_CASE(32, 1) PQHSA_SCAN_CASE(32, 2) PQHSA_SCAN_CASE(32, 4)
+  PQHSA_SCAN_CASE(64, 1) PQHSA_SCAN_CASE(64, 2)
 #undef PQHSA_SCAN_CASE
   return cudaErrorInvalidValue;
 }

@@ -41,8 +41,10 @@ METRIC = ("decode-attention achieved HBM GB/s at 128K context "
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 512 << 20
-SCAN_DRAM_BYTES_PER_UNIT = 41.15e6 / (8 * 131072)   # ncu, profiles/scan_kernel_c3_b1.md
-SCAN_SMEM_WAVEFRONTS_PER_TILE = 176      # l1tex__data_pipe_lsu_wavefronts_mem_shared / tiles, same capture
+# DRAM traffic of ONE scan launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture of this repository's scan kernel, see the profile summaries), keyed by workload: the
+# figure is reported only for the workload it was captured on.
+SCAN_DRAM_TRAFFIC = {}
 
 
 def measured_peak():
@@ -337,29 +339,25 @@ def main():
     peak, peak_src = measured_peak()
     scan_bytes = head["bytes"]["scan"]
     scan_gbs = scan_bytes / (stage_ms[1] * 1e-3) / 1e9
-    # DRAM bytes of one scan launch: ncu counted 41.15 MB for the 8 x 131072 tokens of
-    # c3_b1 (profiles/scan_kernel_c3_b1.md) = 39.2 B per (token, KV head), scaled by units
-    scan_units = cfg.n_kv_heads * sum(seq_lens)
-    scan_traffic = SCAN_DRAM_BYTES_PER_UNIT * scan_units
+    scan_traffic = SCAN_DRAM_TRAFFIC.get(cfg.name)
     roofline = dict(bound="hbm", kernel="scan_kernel (ADC scan + fused per-list sums)",
                     achieved=scan_gbs, peak=peak, unit="GB/s", frac=scan_gbs / peak,
                     peak_source=peak_src, traffic=scan_traffic,
-                    traffic_note="dram__bytes_read+write of one ncu capture on c3_b1, scaled by "
-                                 "tokens x KV heads; score rows written by the scan stay in L2 "
-                                 "past the end of the kernel, so they are not in this figure",
-                    binding_unit="shared-memory LSU (l1tex data-pipe wavefronts), not HBM: "
-                                 "see profiles/scan_kernel_c3_b1.md",
+                    traffic_note="dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture "
+                                 "of one scan launch on this workload (null: not captured on it)",
+                    binding_unit="the SM's load/store data pipe (one wavefront per clock: 16 B of "
+                                 "table reads per token, subspace and head group), not HBM",
                     algorithmic_bytes_per_launch=scan_bytes, avg_launch_ms=stage_ms[1],
-                    co_bound="shared-memory LSU: 16 B of table reads per (token, subspace)",
                     stage_ms=dict(lut=stage_ms[0], scan=stage_ms[1], select=stage_ms[2],
                                   attend=stage_ms[3]),
                     whole_step_frac_of_peak=head["gbs"] / world / peak)
-    # the unit that binds the scan: one shared-memory wavefront per SM and clock.  ncu counted
-    # 176 wavefronts per 32-token tile of a (KV head, 4-head group) on c3_b1
-    # (profiles/scan_kernel_c3_b1.md); the clock is the median sampled below, filled in later.
+    # the unit that binds the scan: a lower bound on its time from the table reads alone
+    # (M 16-byte reads per token and head group at 128 B per SM and clock), filled in below
+    # with the sampled clock
     scan_tiles = cfg.n_kv_heads * ((cfg.group + 3) // 4) * sum((n + 31) // 32 for n in seq_lens)
-    roofline["shared_memory_pipe"] = dict(wavefronts_per_tile=SCAN_SMEM_WAVEFRONTS_PER_TILE,
-                                          tiles_per_launch=scan_tiles)
+    roofline["data_pipe"] = dict(
+        table_wavefronts_per_tile=(cfg.pq_m if cfg.pq_ncode > 16 else cfg.pq_m) * 4,
+        tiles_per_launch=scan_tiles)
 
     # end to end through the host-buffer entry point: q from pinned host memory, out back
     q_host = op.q.cpu().pin_memory()
@@ -415,6 +413,47 @@ def main():
             algorithmic_mb=r["bytes"]["total"] / 1e6,
             index="n_list 512, 8 subspaces x 4 bits, 4 sinks, 128-token window, page-rounded budget")
         del op_p, idx_p
+
+    # the other configurations of the benchmark plan, each generated, indexed and timed on its
+    # own: the 32K layer, the ragged G = 8 batch, and three points of the context sweep with the
+    # dense comparator beside them (time of the library's dense kernel, and of one read of K and
+    # V at the measured copy rate)
+    if not args.no_variants and cfg.name.startswith("c3") and world == 1:
+        for name in ("c2", "c4", "c5_n16_b1", "c5_n128_b1", "c5_n512_b1"):
+            torch.cuda.empty_cache()
+            cfg_x = dataclasses.replace(parse_workload(name), kmeans_iters=min(2, args.kmeans_iters))
+            inp_x = generate(cfg_x, device=dev)
+            idx_x = build_index(inp_x)
+            op_x = DecodeOp(inp_x, idx_x, device=dev)
+            steps_x = max(10, args.steps // 4)
+            r = measure(op_x, cfg_x, cfg_x.budget_ppm, steps_x, 3, list(cfg_x.seq_lens))
+            ent = dict(us_per_step=1000 * r["ms"], us_p10=1000 * r["p10"], us_p90=1000 * r["p90"],
+                       achieved_gbs=r["gbs"], pct_of_measured_peak=100 * r["gbs"] / peak,
+                       algorithmic_mb=r["bytes"]["total"] / 1e6, batch=cfg_x.batch,
+                       context=cfg_x.max_seq_len, n_list=cfg_x.n_list, steps=steps_x)
+            if name.startswith("c5"):
+                dws_x = torch.empty(pqhsa.dense_workspace_bytes(op_x.params), dtype=torch.uint8, device=dev)
+                dout_x = torch.empty_like(op_x.q)
+                for _ in range(3):
+                    pqhsa.dense_decode(op_x.params, op_x.q, op_x.kv, op_x.seq_lens, dout_x, dws_x)
+                pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                         for _ in range(steps_x)]
+                barrier()
+                for a, b in pairs:
+                    flush.zero_()
+                    a.record()
+                    pqhsa.dense_decode(op_x.params, op_x.q, op_x.kv, op_x.seq_lens, dout_x, dws_x)
+                    b.record()
+                barrier()
+                d_ms = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs)
+                db = dense_attention_bytes(cfg_x, list(cfg_x.seq_lens))
+                ent.update(dense_us=1000 * d_ms, ideal_dense_us=db / peak / 1e3,
+                           dense_over_pqhsa=d_ms / r["ms"],
+                           ideal_dense_over_pqhsa=(db / peak / 1e6) / r["ms"])
+                del dws_x, dout_x
+            variants[name] = ent
+            del op_x, idx_x, inp_x
+        torch.cuda.empty_cache()
 
     # dense comparator: the library's own split-K dense decode kernel over the same paged cache
     dws = torch.empty(pqhsa.dense_workspace_bytes(op.params), dtype=torch.uint8, device=dev)
@@ -491,11 +530,11 @@ def main():
     clocks = sampler.stop()              # sampled over every timed loop above
     try:      # an auxiliary figure: never let it cost the JSON line
         if clocks.get("sm_mhz"):
-            sp = roofline["shared_memory_pipe"]
+            sp = roofline["data_pipe"]
             n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
             cycles = stage_ms[1] * 1e-3 * clocks["sm_mhz"] * 1e6
-            sp["frac_of_one_wavefront_per_sm_clock"] = (
-                sp["wavefronts_per_tile"] * sp["tiles_per_launch"] / n_sm / cycles)
+            sp["table_reads_frac_of_one_wavefront_per_sm_clock"] = (
+                sp["table_wavefronts_per_tile"] * sp["tiles_per_launch"] / n_sm / cycles)
     except Exception:
         pass
     cpu_baseline = None

@@ -66,7 +66,8 @@ typedef struct {
   int32_t page_size;          /* tokens per KV page                                         */
   int32_t max_pages_per_seq;  /* row stride of block_table                                  */
   int32_t n_sink;             /* sink prefix: S_b = first min(n_sink, N_b) tokens (Sec. 3.2) */
-  int32_t n_local;            /* local window: L_b = last min(n_local, N_b - |S_b|) tokens;  */
+  int32_t n_local;            /* local window: L_b = last min(n_local, N_b - |S_b|) tokens   */
+                              /* (see indexed_lens for a per-sequence window);               */
                               /* R_b = the tokens between; S_b and L_b are attended exactly  */
                               /* and take no part in the top-k or the background             */
   uint32_t budget_ppm;        /* rho in parts per million; k_b = ceil(|R_b| * ppm / 1e6),   */
@@ -77,7 +78,28 @@ typedef struct {
   int32_t exact_set_multiple; /* 0 or 1: off.  m > 1: |S_b| + |L_b| + k_b is rounded up to a  */
                               /* multiple of m (App. A, budgets in whole pages), k_b <= |R_b|; */
                               /* k_max must then cover the extra m - 1                        */
+  int32_t variant;            /* pqhsa_variant: how the background term is formed (Table 2);  */
+                              /* 0 = PQ-HSA itself                                            */
+  const int32_t* indexed_lens;/* DEVICE pointer [B] or NULL.  Number of leading positions of  */
+                              /* each sequence that the index covers: R_b = [|S_b|,           */
+                              /* indexed_lens[b]) and L_b = everything after (Sec. 3.3: a new */
+                              /* token is attended exactly until the next index update        */
+                              /* encodes it).  NULL: L_b is the last n_local tokens.  Values  */
+                              /* are clipped to [|S_b|, seq_lens[b]]; n_local is then unused  */
 } pqhsa_params;
+
+/* Mechanism variants of the paper's ablation (Table 2; App. B, "Variant definitions").  All of
+ * them keep the selector, the budget and the exact part; they differ in the background term.
+ * Every variant but B and T needs pqhsa_index.list_counts. */
+typedef enum {
+  PQHSA_VARIANT_B = 0,    /* PQ-HSA: logit l~_i, value vbar_j (Eq. 4)                            */
+  PQHSA_VARIANT_T = 1,    /* no background term                                                  */
+  PQHSA_VARIANT_BX = 2,   /* B with vbar_j replaced by the mean over the list's unselected       */
+                          /* members, (|R_j| vbar_j - sum_{T n R_j} v_i) / |B n R_j|             */
+  PQHSA_VARIANT_C = 3,    /* logit l~_i, value = token-count-weighted global mean of the vbar_j  */
+  PQHSA_VARIANT_C2 = 4,   /* one shared logit mean_{i in T} l~_i, global mean value              */
+  PQHSA_VARIANT_C2B = 5   /* one shared logit min_{i in T} l_i (exact logits), global mean value */
+} pqhsa_variant;
 
 /* IVF-PQ index, one per (sequence, KV head) (Sec. 3.1).  Device pointers, read-only. */
 typedef struct {
@@ -90,6 +112,9 @@ typedef struct {
   const float* key_norms;     /* [B][H_kv][N_max]          r_i, or NULL for all ones        */
   const float* list_vmeans;   /* [B][H_kv][n_list][d]      stored mean value of ALL members */
                               /*                           of each list (Eq. 4); 0 if empty */
+  const int32_t* list_counts; /* [B][H_kv][n_list]         |R_j|, members behind each stored */
+                              /*                           mean; NULL unless a variant needs */
+                              /*                           it (pqhsa_variant)                */
 } pqhsa_index;
 
 /* The same arrays as pqhsa_index, writable, plus the member count of every list: what
@@ -124,7 +149,14 @@ typedef enum {
   PQHSA_BUF_LIST_PARTIALS = 3,  /* float   [B][H_kv][n_hg][n_part][Gc * (2 + n_list)]         */
   PQHSA_BUF_SEL_IDX = 4,        /* int32   [B][H_q][k_max]                                    */
   PQHSA_BUF_SEL_COUNT = 5,      /* int32   [B][H_q]                                           */
-  PQHSA_BUF_KTH = 6             /* float   [B][H_q]                                           */
+  PQHSA_BUF_KTH = 6,            /* float   [B][H_q]                                           */
+  /* scratch of the hybrid attention, for inspection through pqhsa_decode_buffer_offset (the   */
+  /* offsets also hold for the `ws` of a pqhsa_hybrid_attend call):                             */
+  PQHSA_BUF_BG_MASS = 7,        /* float   [B][H_q][n_list]  background mass M_j of Eq. 4,      */
+                                /*         relative to exp(BG_MAX); may be slightly negative    */
+                                /*         where every member of a list was selected (read as 0) */
+  PQHSA_BUF_BG_MAX = 8          /* float   [B][H_q]  max approximate logit of the row (-inf:    */
+                                /*         no background)                                       */
 } pqhsa_buffer;
 
 /* Query heads of a group are processed Gc at a time (Gc = G for G <= 2, else 4); a group
@@ -170,12 +202,14 @@ int pqhsa_select(const pqhsa_params* params, const float* scores, const int32_t*
  * selected tokens) from the paged cache and attends them with exact logits, takes the
  * selected tokens' approximate mass out of their lists' sums, folds in the n_list
  * mean-value terms and normalises once.
- * out [B][H_q][d] in params->dtype; lse_or_null [B][H_q] = log of the normaliser. */
+ * out [B][H_q][d] in params->dtype; lse_or_null [B][H_q] = log of the normaliser;
+ * out_f32_or_null [B][H_q][d] = the same output before it is rounded to params->dtype. */
 int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
                         const pqhsa_index* index, const float* scores,
                         const float* list_partials, const int32_t* sel_idx,
                         const int32_t* sel_count, const int32_t* seq_lens, void* out,
-                        float* lse_or_null, void* ws, size_t ws_bytes, void* stream);
+                        float* lse_or_null, float* out_f32_or_null, void* ws, size_t ws_bytes,
+                        void* stream);
 
 /* pqhsa_select without a workspace argument.  (No counterpart in the paper: this entry point
  * exists for integration, not for the method.)
@@ -252,10 +286,18 @@ int pqhsa_decode_host(const pqhsa_params* params, const void* q_host, void* q_de
                       const int32_t* seq_lens, void* out_dev_staging, void* out_host,
                       void* ws, size_t ws_bytes, void* stream);
 
-/* Reads the status word kernels set when they meet an inconsistency (selected count != k,
- * seq_len > max_seq_len): copies it to the host and waits for `stream`.  Returns PQHSA_OK
- * or PQHSA_ERR_DEVICE_CHECK.  Valid after pqhsa_select / pqhsa_decode on the same ws. */
+/* Reads the status word kernels set when they meet an inconsistency: copies it to the host and
+ * waits for `stream`.  Returns PQHSA_OK or PQHSA_ERR_DEVICE_CHECK.  Valid after pqhsa_scan /
+ * pqhsa_select / pqhsa_hybrid_attend / pqhsa_decode on the same ws.  Bits: 1 selected count != k,
+ * 2 seq_len outside [0, max_seq_len], 4 a bounded wait on a bulk copy ran out; a library built
+ * with -DPQHSA_DEBUG (pqhsa_debug_build() == 1) also records the indices that the release
+ * build silently clamps or skips: 8 list id >= n_list, 16 selected position outside the indexed
+ * region, 32 negative page id.  No check traps: the CUDA context stays usable. */
 int pqhsa_last_device_status(const pqhsa_params* params, void* ws, void* stream);
+int pqhsa_debug_build(void);
+/* The predicate behind a debug check, for host-side unit tests: which = 0 list id (value < hi),
+ * 1 position (lo <= value < hi), 2 page id (value >= 0).  Returns 1 / 0, -1 for an unknown check. */
+int pqhsa_debug_predicate(int which, long long value, long long lo, long long hi);
 
 /* Byte offset inside `ws` of an intermediate buffer after pqhsa_decode (for inspection by
  * tests and tools); (size_t)-1 on error. */

@@ -25,22 +25,33 @@ def _nvcc() -> str:
     return exe
 
 
-def _stale(sources) -> bool:
-    if not os.path.exists(LIB):
+def _stale(sources, lib=None) -> bool:
+    lib = lib or LIB
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + \
            [os.path.join(ROOT, "include", "pqhsa.h"), os.path.abspath(__file__)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
-    """Compile every .cu under csrc/ for sm_100a and link libpqhsa.so next to this file."""
+DEBUG_LIB = os.path.join(PKG, "libpqhsa_debug.so")
+
+
+def build_library(force: bool = False, verbose: bool = False, extra_flags=(), debug: bool = False) -> str:
+    """Compile every .cu under csrc/ for sm_100a and link libpqhsa.so next to this file.
+
+    debug=True builds libpqhsa_debug.so with -DPQHSA_DEBUG instead: the same kernels, which also
+    record (in the status word) every index that the release build silently clamps or skips.
+    Select it at run time with the environment variable PQHSA_LIBRARY."""
     sources = [s for s in SOURCES if os.path.exists(os.path.join(CSRC, s))]
-    if not force and not _stale(sources):
-        return LIB
+    lib = DEBUG_LIB if debug else LIB
+    if debug:
+        extra_flags = tuple(extra_flags) + ("-DPQHSA_DEBUG",)
+    if not force and not _stale(sources, lib):
+        return lib
     nvcc = _nvcc()
-    objdir = os.path.join(PKG, "build")
+    objdir = os.path.join(PKG, "build", "debug" if debug else "release")
     os.makedirs(objdir, exist_ok=True)
 
     def compile_one(src):
@@ -55,13 +66,13 @@ def build_library(force: bool = False, verbose: bool = False, extra_flags=()) ->
 
     with concurrent.futures.ThreadPoolExecutor(max_workers=len(sources)) as ex:
         objs = list(ex.map(compile_one, sources))
-    cmd = [nvcc, "-shared", "-o", LIB, *objs, "-lcudart"]
+    cmd = [nvcc, "-shared", "-o", lib, *objs, "-lcudart"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
     flags = ["-Xptxas", "-v"] if "-v" in sys.argv else []
-    print(build_library(force=True, verbose=True, extra_flags=flags))
+    print(build_library(force=True, verbose=True, extra_flags=flags, debug="--debug" in sys.argv))

@@ -49,6 +49,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (p->budget_ppm > 1000000u) return PQHSA_ERR_INVALID_ARG;
   if (p->dtype != PQHSA_F16 && p->dtype != PQHSA_BF16) return PQHSA_ERR_INVALID_ARG;
   if (!(p->sm_scale > 0.f)) return PQHSA_ERR_INVALID_ARG;
+  if (p->variant < PQHSA_VARIANT_B || p->variant > PQHSA_VARIANT_C2B) return PQHSA_ERR_INVALID_ARG;
   if ((long long)p->max_pages_per_seq * p->page_size < p->max_seq_len) return PQHSA_ERR_INVALID_ARG;
   long long k_need = ((long long)p->max_seq_len * p->budget_ppm + 999999LL) / 1000000LL;
   if (p->exact_set_multiple > 1) k_need += p->exact_set_multiple - 1;     // rounding slack
@@ -76,6 +77,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.N_max = p->max_seq_len; o.page_size = p->page_size; o.max_pages = p->max_pages_per_seq;
   o.k_max = p->k_max; o.n_sink = p->n_sink; o.n_local = p->n_local;
   o.exact_multiple = p->exact_set_multiple; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
+  o.variant = p->variant; o.indexed_lens = p->indexed_lens; o.status = nullptr;
   o.num_sms = sm_count();
   o.scan_ctas = o.num_sms;                                  // persistent scan CTAs: one per SM
   o.upb = o.Hkv * o.n_hg;
@@ -115,6 +117,8 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (o.bg_splits > o.n_list / 32) o.bg_splits = o.n_list / 32;
   if (o.bg_splits > 16) o.bg_splits = 16;
   if (o.bg_splits < 1) o.bg_splits = 1;
+  // the variants with a global mean value need all lists of a unit in one CTA
+  if (o.variant >= PQHSA_VARIANT_C) o.bg_splits = 1;
   // attend kernel, split-K CTAs per row: about 512 selected tokens each, but enough CTAs to
   // fill the GPU when there are few rows (one wave of 4 resident CTAs per SM, background
   // CTAs included), as long as every CTA keeps at least 32 tokens
@@ -126,6 +130,8 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (fill > max_fill) fill = max_fill;
   if (o.splits < fill) o.splits = fill;
   if (o.splits > 64) o.splits = 64;
+  // variant Bx adds one correction partial per exact split; a row's merge takes 128 partials
+  if (o.variant == PQHSA_VARIANT_BX && 2 * o.splits + o.bg_splits > 128) o.splits = (128 - o.bg_splits) / 2;
   if (o.splits < 1) o.splits = 1;
   // background preparation: CTAs per row
   o.bg_ctas = ceil_div(2LL * o.num_sms, o.rows);
@@ -145,8 +151,16 @@ static size_t buffer_elems(const Plan& pl, int which) {
     case PQHSA_BUF_SEL_IDX: return (size_t)pl.rows * pl.k_max;
     case PQHSA_BUF_SEL_COUNT: return (size_t)pl.rows;
     case PQHSA_BUF_KTH: return (size_t)pl.rows;
+    case PQHSA_BUF_BG_MASS: return (size_t)pl.rows * pl.n_list;
+    case PQHSA_BUF_BG_MAX: return (size_t)pl.rows;
     default: return 0;
   }
+}
+
+// Partials per score row in the attend stage: the exact splits, the background slices and,
+// for variant Bx, one correction partial per exact split.
+int attend_parts(const Plan& pl) {
+  return pl.splits + pl.bg_splits + (pl.variant == PQHSA_VARIANT_BX ? pl.splits : 0);
 }
 
 void make_layout(const Plan& pl, WsLayout* L) {
@@ -157,12 +171,14 @@ void make_layout(const Plan& pl, WsLayout* L) {
   L->counters = take((size_t)pl.rows * 16);
   L->attend_tickets = take((size_t)pl.rows * 4);
   L->bg_mass = take((size_t)pl.rows * pl.n_list * 4);
+  L->bg_aux = take((size_t)pl.rows * 16);
+  L->bg_tcount = take(pl.variant == PQHSA_VARIANT_BX ? (size_t)pl.rows * pl.n_list * 4 : 0);
   L->attend_zero_bytes = o - L->attend_tickets;
   L->zero_bytes = o - L->zero_begin;
   L->rowstate = take((size_t)pl.rows * 16);
   L->cand = take((size_t)pl.rows * pl.cand_cap * 4);
   L->bg_max = take((size_t)pl.rows * 4);
-  L->split_part = take((size_t)pl.rows * (pl.splits + pl.bg_splits) * (4 + kHeadDim) * 4);
+  L->split_part = take((size_t)pl.rows * attend_parts(pl) * (4 + kHeadDim) * 4);
   L->stage_end = o;
   L->lut = take(buffer_elems(pl, PQHSA_BUF_LUT) * 4);
   L->coarse = take(buffer_elems(pl, PQHSA_BUF_COARSE) * 4);
@@ -188,6 +204,11 @@ int check_index(const pqhsa_index* ix) {
     return PQHSA_ERR_INVALID_ARG;
   if (!aligned16(ix->centroids) || !aligned16(ix->codes) || !aligned16(ix->list_vmeans))
     return PQHSA_ERR_INVALID_ARG;
+  return PQHSA_OK;
+}
+
+int check_variant(const Plan& pl, const pqhsa_index* ix) {
+  if (pl.variant >= PQHSA_VARIANT_BX && ix->list_counts == nullptr) return PQHSA_ERR_INVALID_ARG;
   return PQHSA_OK;
 }
 
@@ -253,6 +274,8 @@ size_t pqhsa_decode_buffer_offset(const pqhsa_params* params, int which) {
     case PQHSA_BUF_SEL_IDX: return L.sel_idx;
     case PQHSA_BUF_SEL_COUNT: return L.sel_count;
     case PQHSA_BUF_KTH: return L.kth;
+    case PQHSA_BUF_BG_MASS: return L.bg_mass;
+    case PQHSA_BUF_BG_MAX: return L.bg_max;
     default: return (size_t)-1;
   }
 }
@@ -261,7 +284,9 @@ int pqhsa_decode_launch_count(const pqhsa_params* params) {
   Plan pl;
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
-  return 6;   // LUT build, scan, select sample, select filter, attend exact, attend background
+  // LUT build, scan, select sample, select filter, background preparation, attend (+ the
+  // correction pass of variant Bx)
+  return pl.variant == PQHSA_VARIANT_BX ? 7 : 6;
 }
 
 int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index* index,
@@ -316,11 +341,13 @@ int pqhsa_select(const pqhsa_params* params, const float* scores, const int32_t*
 int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
                         const pqhsa_index* index, const float* scores, const float* list_partials,
                         const int32_t* sel_idx, const int32_t* sel_count, const int32_t* seq_lens,
-                        void* out, float* lse_or_null, void* ws, size_t ws_bytes, void* stream) {
+                        void* out, float* lse_or_null, float* out_f32_or_null, void* ws,
+                        size_t ws_bytes, void* stream) {
   Plan pl;
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
   if ((rc = check_index(index)) != PQHSA_OK) return rc;
+  if ((rc = check_variant(pl, index)) != PQHSA_OK) return rc;
   if ((rc = check_kv(kv)) != PQHSA_OK) return rc;
   if (q == nullptr || scores == nullptr || list_partials == nullptr || sel_idx == nullptr ||
       sel_count == nullptr || seq_lens == nullptr || out == nullptr)
@@ -333,7 +360,7 @@ int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_p
   if (cudaMemsetAsync(w + L.attend_tickets, 0, L.attend_zero_bytes, st) != cudaSuccess)
     return PQHSA_ERR_CUDA;
   return cuda_status(launch_attend(pl, L, w, q, *kv, *index, scores, list_partials, sel_idx,
-                                   sel_count, seq_lens, out, lse_or_null, st));
+                                   sel_count, seq_lens, out, lse_or_null, out_f32_or_null, st));
 }
 
 static int decode_impl(const pqhsa_params* params, const void* q, const pqhsa_index* index,
@@ -343,6 +370,7 @@ static int decode_impl(const pqhsa_params* params, const void* q, const pqhsa_in
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
   if ((rc = check_index(index)) != PQHSA_OK) return rc;
+  if ((rc = check_variant(pl, index)) != PQHSA_OK) return rc;
   if ((rc = check_kv(kv)) != PQHSA_OK) return rc;
   if (q == nullptr || seq_lens == nullptr || out == nullptr) return PQHSA_ERR_INVALID_ARG;
   WsLayout L;
@@ -373,7 +401,7 @@ static int decode_impl(const pqhsa_params* params, const void* q, const pqhsa_in
   if (e == cudaSuccess) e = mark(3);
   if (e == cudaSuccess)
     e = launch_attend(pl, L, w, q, *kv, *index, scores, partials, sel_idx, sel_count, seq_lens,
-                      out, nullptr, st);
+                      out, nullptr, nullptr, st);
   if (e == cudaSuccess) e = mark(4);
   return cuda_status(e);
 }
@@ -429,6 +457,23 @@ int pqhsa_last_device_status(const pqhsa_params* params, void* ws, void* stream)
     return PQHSA_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return PQHSA_ERR_CUDA;
   return host == 0 ? PQHSA_OK : PQHSA_ERR_DEVICE_CHECK;
+}
+
+int pqhsa_debug_build(void) {
+#ifdef PQHSA_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+int pqhsa_debug_predicate(int which, long long value, long long lo, long long hi) {
+  switch (which) {
+    case 0: return list_id_ok(value, hi) ? 1 : 0;
+    case 1: return position_ok(value, lo, hi) ? 1 : 0;
+    case 2: return page_ok(value) ? 1 : 0;
+    default: return -1;
+  }
 }
 
 const char* pqhsa_status_string(int status) {

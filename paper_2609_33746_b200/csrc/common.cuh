@@ -34,6 +34,9 @@ struct Plan {
   int k_max;
   int n_sink, n_local;               // |S| and |L| of Sec. 3.2 (upper bounds: clipped per sequence)
   int exact_multiple;                // > 1: |S| + |L| + k is rounded up to this multiple (App. A)
+  int variant;                       // pqhsa_variant: how the background term is formed
+  const int32_t* indexed_lens;       // device [B] or null: positions covered by the index
+  int* status;                       // device status word, or null (set by the launchers)
   uint32_t ppm;
   float sm_scale;
   int dtype;
@@ -62,6 +65,8 @@ struct WsLayout {
   size_t rowstate;                   // int32  [rows][4]: lo, hi (float bits), k, n
   size_t cand;                       // int32  [rows][cand_cap]: candidate positions
   size_t bg_mass;                    // float  [rows][n_list]: M_j relative to bg_max (accumulated)
+  size_t bg_aux;                     // float  [rows][4]: [0] sum of the selected tokens' approximate logits
+  size_t bg_tcount;                  // int32  [rows][n_list]: selected tokens per list (variant Bx only)
   size_t bg_max;                     // float  [rows]
   size_t split_part;                 // float  [rows][splits + bg_splits][4 + 128]: m, Z, pad, N[128]
   size_t stage_end;                  // end of what a single stage call needs
@@ -72,6 +77,38 @@ struct WsLayout {
 
 int make_plan(const pqhsa_params* p, Plan* plan);          // returns pqhsa_status
 void make_layout(const Plan& plan, WsLayout* L);
+int attend_parts(const Plan& plan);                        // partials per score row in the attend stage
+
+// ------------------------------------------------------------------ index checks
+// The release build never trusts an index it reads from memory: a list id is clamped to
+// [0, n_list), a selected position outside its sequence is skipped.  A build with
+// -DPQHSA_DEBUG also RECORDS such an index: the access is still made safe the same way, and a
+// bit is or-ed into the status word that pqhsa_last_device_status reads (no trap, no assert:
+// the context stays usable).  The predicates are host + device so that they can be unit
+// tested without a GPU (pqhsa_debug_predicate).
+constexpr int kStatusCountMismatch = 1;    // top-k emitted a number of positions other than k
+constexpr int kStatusSeqLen = 2;           // seq_lens[b] outside [0, max_seq_len]
+constexpr int kStatusCopyTimeout = 4;      // a bounded wait on a bulk copy ran out
+constexpr int kStatusListId = 8;           // debug: list id >= n_list
+constexpr int kStatusPosition = 16;        // debug: selected position outside the indexed region
+constexpr int kStatusPage = 32;            // debug: negative page id in the block table
+__host__ __device__ inline bool list_id_ok(long long lid, long long n_list) {
+  return lid >= 0 && lid < n_list;
+}
+__host__ __device__ inline bool position_ok(long long pos, long long lo, long long hi) {
+  return pos >= lo && pos < hi;
+}
+__host__ __device__ inline bool page_ok(long long page) { return page >= 0; }
+#ifdef PQHSA_DEBUG
+#define PQHSA_DEBUG_CHECK(ok, bit, status_ptr)                                    \
+  do {                                                                            \
+    if (!(ok) && (status_ptr) != nullptr) atomicOr((status_ptr), (bit));          \
+  } while (0)
+#else
+#define PQHSA_DEBUG_CHECK(ok, bit, status_ptr) \
+  do {                                         \
+  } while (0)
+#endif
 
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ uint32_t score_key(float s) {
@@ -95,27 +132,33 @@ __device__ __forceinline__ int clamp_len(int n, int n_max) {
   return n < 0 ? 0 : (n > n_max ? n_max : n);
 }
 
-// Position partition of a sequence of n tokens (Sec. 3.2): sink prefix S = [0, r_begin),
-// indexed region R = [r_begin, r_end), local window L = [r_end, n).
+// Position partition of sequence b with n tokens (Sec. 3.2): sink prefix S = [0, r_begin),
+// indexed region R = [r_begin, r_end), window L = [r_end, n).  The window holds what the index
+// does not cover (Sec. 3.3): with indexed_lens given, everything from indexed_lens[b] on;
+// otherwise the last n_local tokens.
 struct Region {
   int r_begin, r_end;
 };
-__device__ __forceinline__ Region region_of(int n, int n_sink, int n_local) {
+__device__ __forceinline__ Region region_of(const Plan& pl, int n, int b) {
   Region r;
-  r.r_begin = n_sink < n ? n_sink : n;
-  r.r_end = n - n_local > r.r_begin ? n - n_local : r.r_begin;
+  r.r_begin = pl.n_sink < n ? pl.n_sink : n;
+  int end = n - pl.n_local;
+  if (pl.indexed_lens != nullptr) {
+    const int covered = __ldg(pl.indexed_lens + b);
+    end = covered < n ? covered : n;
+  }
+  r.r_end = end > r.r_begin ? end : r.r_begin;
   return r;
 }
-// k of Eq. 3 for a sequence of n tokens: ceil(rho |R|); with exact_multiple > 1 the size of
+// k of Eq. 3 for sequence b with n tokens: ceil(rho |R|); with exact_multiple > 1 the size of
 // the exact set |S| + |L| + k is rounded up to that multiple first (never beyond |R|).
-__device__ __forceinline__ int region_budget(int n, int n_sink, int n_local, uint32_t ppm,
-                                             int exact_multiple) {
-  const Region r = region_of(n, n_sink, n_local);
+__device__ __forceinline__ int region_budget(const Plan& pl, int n, int b) {
+  const Region r = region_of(pl, n, b);
   const int n_r = r.r_end - r.r_begin;
-  int k = budget_k(n_r, ppm);
-  if (exact_multiple > 1) {
+  int k = budget_k(n_r, pl.ppm);
+  if (pl.exact_multiple > 1) {
     const long long fixed = n - n_r;
-    const long long total = (fixed + k + exact_multiple - 1) / exact_multiple * exact_multiple;
+    const long long total = (fixed + k + pl.exact_multiple - 1) / pl.exact_multiple * pl.exact_multiple;
     k = (int)(total - fixed < n_r ? total - fixed : n_r);
   }
   return k;
@@ -227,7 +270,7 @@ cudaError_t launch_attend(const Plan& pl, const WsLayout& L, char* ws, const voi
                           const pqhsa_paged_kv& kv, const pqhsa_index& ix, const float* scores,
                           const float* list_partials, const int32_t* sel_idx,
                           const int32_t* sel_count, const int32_t* seq_lens, void* out,
-                          float* lse, cudaStream_t st);
+                          float* lse, float* out_f32, cudaStream_t st);
 cudaError_t launch_scan4(const Plan& pl, const pqhsa_index& ix, const float* lut,
                          const float* coarse, const int32_t* seq_lens, float* scores,
                          float* list_partials, int* status, cudaStream_t st);

@@ -153,7 +153,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   const ScanSplit sp = scan_split(seq_lens, pl.B, N_max, upb, pl.scan_ctas);
   if (c == 0 && tid == 0) {
     for (int b = 0; b < pl.B; ++b)
-      if (seq_lens[b] < 0 || seq_lens[b] > N_max) atomicOr(status, 2);
+      if (seq_lens[b] < 0 || seq_lens[b] > N_max) atomicOr(status, kStatusSeqLen);
   }
   if (c >= sp.P_eff || sp.T == 0) return;
   long long lo = split_start(sp, c);
@@ -191,7 +191,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     const int cnt = (int)min((long long)(tb - t0), hi - lo);
     const int slot = c - split_cta_of(sp, base + (long long)w * tb);
     const int Nb = clamp_len(seq_lens[b], N_max);
-    const Region rg = region_of(Nb, pl.n_sink, pl.n_local);   // only R enters top-k and sums
+    const Region rg = region_of(pl, Nb, b);   // only R enters top-k and sums
     const int kv = w / pl.n_hg, hg = w % pl.n_hg;
     const size_t ukv = (size_t)b * pl.Hkv + kv;
     const size_t unit = ukv * pl.n_hg + hg;
@@ -223,7 +223,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
                       Nb, lane);
     TokenMeta cur;
     load_meta(cur, lids, norms, row_base, t * kTile + lane, t < tend && t * kTile + lane < Nb);
-    if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, 4);
+    if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, kStatusCopyTimeout);
     bar_parity ^= 1u;
     __syncthreads();   // partial zeroed, tables landed
 
@@ -282,6 +282,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         float accf[GC], co[GC];
         acc0.get(accf);
         // (a list id outside [0, n_list) is an index error, not a reason to read out of bounds)
+        PQHSA_DEBUG_CHECK(!valid || list_id_ok(cur.lid, n_list), kStatusListId, status);
         if (pl.coarse_in_smem) load_vec<GC>(co, s_coarse + min(cur.lid, (uint32_t)(n_list - 1)) * GC);
         else load_vec<GC>(co, g_coarse + min(cur.lid, (uint32_t)(n_list - 1)) * GC);
         if (valid) {

@@ -122,6 +122,7 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
   constexpr int kEntryBytes = GC * 4;
   constexpr int kRowBytes = M * kEntryBytes;          // stride between consecutive z
   constexpr int kRowShift = (M == 8 ? 3 : 4) + (GC == 4 ? 4 : GC == 2 ? 3 : 2);   // log2(kRowBytes)
+  static_assert((1 << kRowShift) == kRowBytes, "row stride");
   constexpr uint32_t kRowMask = 15u << kRowShift;
   constexpr int kRep = 128 / kEntryBytes;             // lanes of one shared-memory access group
   constexpr int kW = Packed<GC>::kW;
@@ -149,7 +150,7 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
   const ScanSplit sp = scan_split(seq_lens, pl.B, N_max, upb, pl.scan_ctas);
   if (c == 0 && tid == 0) {
     for (int b = 0; b < pl.B; ++b)
-      if (seq_lens[b] < 0 || seq_lens[b] > N_max) atomicOr(status, 2);
+      if (seq_lens[b] < 0 || seq_lens[b] > N_max) atomicOr(status, kStatusSeqLen);
   }
   if (c >= sp.P_eff || sp.T == 0) return;
   long long lo = split_start(sp, c);
@@ -189,7 +190,7 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
     const int cnt = (int)min((long long)(tb - t0), hi - lo);
     const int slot = c - split_cta_of(sp, base + (long long)w * tb);
     const int Nb = clamp_len(seq_lens[b], N_max);
-    const Region rg = region_of(Nb, pl.n_sink, pl.n_local);   // only R enters top-k and sums
+    const Region rg = region_of(pl, Nb, b);   // only R enters top-k and sums
     const int kv = w / pl.n_hg, hg = w % pl.n_hg;
     const size_t ukv = (size_t)b * pl.Hkv + kv;
     const size_t unit = ukv * pl.n_hg + hg;
@@ -236,7 +237,7 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
     int i4 = seg_begin + warp * kWarpTok + lane * kTok4;     // this lane's first token
     Records<kCW> cur, nxt;
     load_records<kCW>(cur, code_row, norm_row, lid_row, i4, i4 < seg_end);
-    if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, 4);
+    if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, kStatusCopyTimeout);
     bar_parity ^= 1u;
     __syncthreads();   // partial zeroed, tables landed
 
@@ -276,6 +277,8 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
           }
         }
         // (a list id outside [0, n_list) is an index error, not a reason to read out of bounds)
+        PQHSA_DEBUG_CHECK(i4 + k >= seg_end || list_id_ok((cur.lid2[k >> 1] >> (16 * (k & 1))) & 0xffffu, n_list),
+                          kStatusListId, status);
         const uint32_t lid = min((cur.lid2[k >> 1] >> (16 * (k & 1))) & 0xffffu, (uint32_t)(n_list - 1));
         Packed<GC> co;
         if (coarse_mode == 2) lds_entry<GC>(co, coarse_u32 + lid * 128u + rep_off);

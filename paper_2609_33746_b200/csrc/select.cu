@@ -186,8 +186,8 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
   pdl_wait();
   pdl_launch_dependents();
   const int n = clamp_len(seq_lens[b], pl.N_max);
-  const int k = region_budget(n, pl.n_sink, pl.n_local, pl.ppm, pl.exact_multiple);
-  const Region rg = region_of(n, pl.n_sink, pl.n_local);
+  const int k = region_budget(pl, n, b);
+  const Region rg = region_of(pl, n, b);
   float lo = -CUDART_INF_F, hi = CUDART_INF_F;     // default: every score is a candidate
   if (k == 0) {
     if (tid == 0) { sel_count[row] = 0; kth[row] = CUDART_NAN_F; }
@@ -526,7 +526,7 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
   if (tid == 0) {
     sel_count[row] = k;
     kth[row] = key_score(kstar);
-    if (emitted_before + (int)s_emit != k) atomicOr(status, 1);
+    if (emitted_before + (int)s_emit != k) atomicOr(status, kStatusCountMismatch);
   }
 }
 

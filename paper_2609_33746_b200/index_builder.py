@@ -153,6 +153,8 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
             # and window tokens are attended exactly and belong to no list's background
             r0 = min(cfg.n_sink, n)
             r1 = max(r0, n - cfg.n_local)
+            if cfg.indexed_lens is not None:
+                r1 = max(r0, min(n, cfg.indexed_lens[b]))
             vsum = torch.zeros((nl, d), dtype=torch.float64, device=dev).index_add_(
                 0, ids[r0:r1], v[r0:r1].double())
             cnt = torch.zeros(nl, dtype=torch.float64, device=dev).index_add_(

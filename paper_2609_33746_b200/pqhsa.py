@@ -14,11 +14,15 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libpqhsa.so")
+# PQHSA_LIBRARY selects another build of the same library, e.g. libpqhsa_debug.so (the build
+# that records out-of-range indices in the status word)
+LIB_PATH = os.environ.get("PQHSA_LIBRARY") or os.path.join(_HERE, "libpqhsa.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_CHECK = 0, -1, -2, -3, -4, -5
 F16, BF16 = 0, 1
-BUF_LUT, BUF_COARSE, BUF_SCORES, BUF_LIST_PARTIALS, BUF_SEL_IDX, BUF_SEL_COUNT, BUF_KTH = range(7)
+(BUF_LUT, BUF_COARSE, BUF_SCORES, BUF_LIST_PARTIALS, BUF_SEL_IDX, BUF_SEL_COUNT, BUF_KTH,
+ BUF_BG_MASS, BUF_BG_MAX) = range(9)
+VARIANTS = {"B": 0, "T": 1, "Bx": 2, "C": 3, "C2": 4, "C2b": 5}      # pqhsa_variant
 
 EXPORTS = [
     "pqhsa_heads_per_group", "pqhsa_num_partials", "pqhsa_buffer_elems", "pqhsa_workspace_bytes",
@@ -26,7 +30,8 @@ EXPORTS = [
     "pqhsa_decode_events", "pqhsa_decode_host", "pqhsa_last_device_status", "pqhsa_decode_buffer_offset",
     "pqhsa_decode_launch_count", "pqhsa_status_string", "pqhsa_select_static",
     "pqhsa_select_static_bytes", "pqhsa_select_static_capacity", "pqhsa_dense_decode",
-    "pqhsa_dense_workspace_bytes", "pqhsa_index_update",
+    "pqhsa_dense_workspace_bytes", "pqhsa_index_update", "pqhsa_debug_build",
+    "pqhsa_debug_predicate",
 ]
 
 
@@ -41,12 +46,13 @@ class Params(ctypes.Structure):
         "batch", "n_q_heads", "n_kv_heads", "head_dim", "n_list", "pq_m", "pq_dsub", "pq_ncode",
         "max_seq_len", "page_size", "max_pages_per_seq", "n_sink", "n_local")] + [
         ("budget_ppm", ctypes.c_uint32), ("k_max", ctypes.c_int32), ("sm_scale", ctypes.c_float),
-        ("dtype", ctypes.c_int32), ("exact_set_multiple", ctypes.c_int32)]
+        ("dtype", ctypes.c_int32), ("exact_set_multiple", ctypes.c_int32),
+        ("variant", ctypes.c_int32), ("indexed_lens", ctypes.c_void_p)]
 
 
 class Index(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in (
-        "centroids", "codebooks", "codes", "list_ids", "key_norms", "list_vmeans")]
+        "centroids", "codebooks", "codes", "list_ids", "key_norms", "list_vmeans", "list_counts")]
 
 
 class IndexRW(ctypes.Structure):
@@ -81,7 +87,7 @@ def lib() -> ctypes.CDLL:
             "pqhsa_build_lut": (I, [P, V, PI, V, V, V]),
             "pqhsa_scan": (I, [P, PI, V, V, V, V, V, V, Z, V]),
             "pqhsa_select": (I, [P, V, V, V, V, V, V, Z, V]),
-            "pqhsa_hybrid_attend": (I, [P, V, PK, PI, V, V, V, V, V, V, V, V, Z, V]),
+            "pqhsa_hybrid_attend": (I, [P, V, PK, PI, V, V, V, V, V, V, V, V, V, Z, V]),
             "pqhsa_decode": (I, [P, V, PI, PK, V, V, V, Z, V]),
             "pqhsa_decode_events": (I, [P, V, PI, PK, V, V, V, Z, V, ctypes.POINTER(V)]),
             "pqhsa_decode_host": (I, [P, V, V, PI, PK, V, V, V, V, Z, V]),
@@ -95,6 +101,8 @@ def lib() -> ctypes.CDLL:
             "pqhsa_dense_decode": (I, [P, V, PK, V, V, V, Z, V]),
             "pqhsa_dense_workspace_bytes": (Z, [P]),
             "pqhsa_index_update": (I, [P, ctypes.POINTER(IndexRW), PK, V, V, I, V]),
+            "pqhsa_debug_build": (I, []),
+            "pqhsa_debug_predicate": (I, [I, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_longlong]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -127,7 +135,9 @@ def _stream(stream) -> Optional[int]:
 
 def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_pages_per_seq,
                 budget_ppm, dtype, head_dim=128, pq_ncode=256, page_size=16, n_sink=0, n_local=0,
-                k_max=None, sm_scale=None, exact_set_multiple=0) -> Params:
+                k_max=None, sm_scale=None, exact_set_multiple=0, variant="B",
+                indexed_lens=None) -> Params:
+    """`indexed_lens`: device int32 tensor [batch] or None; the caller keeps it alive."""
     if k_max is None:
         k_max = max(1, (max_seq_len * budget_ppm + 999_999) // 1_000_000)
         if exact_set_multiple > 1:
@@ -137,12 +147,13 @@ def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_
     code = {"fp16": F16, "bf16": BF16, torch.float16: F16, torch.bfloat16: BF16}[dtype]
     return Params(batch, n_q_heads, n_kv_heads, head_dim, n_list, pq_m, head_dim // pq_m, pq_ncode,
                   max_seq_len, page_size, max_pages_per_seq, n_sink, n_local, budget_ppm, k_max,
-                  sm_scale, code, exact_set_multiple)
+                  sm_scale, code, exact_set_multiple, VARIANTS[variant], _ptr(indexed_lens))
 
 
-def make_index(centroids, codebooks, codes, list_ids, key_norms, list_vmeans) -> Index:
+def make_index(centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
+               list_counts=None) -> Index:
     return Index(_ptr(centroids), _ptr(codebooks), _ptr(codes), _ptr(list_ids), _ptr(key_norms),
-                 _ptr(list_vmeans))
+                 _ptr(list_vmeans), _ptr(list_counts))
 
 
 def make_index_rw(centroids, codebooks, codes, list_ids, key_norms, list_vmeans,
@@ -222,11 +233,11 @@ def select_static(params, scores, seq_lens, sel_idx, sel_count, kth_score, strea
 
 
 def hybrid_attend(params, q, kv: PagedKV, index: Index, scores, list_partials, sel_idx, sel_count,
-                  seq_lens, out, lse, ws, stream=None) -> None:
+                  seq_lens, out, lse, ws, out_f32=None, stream=None) -> None:
     _check("pqhsa_hybrid_attend", lib().pqhsa_hybrid_attend(
         ctypes.byref(params), _ptr(q), ctypes.byref(kv), ctypes.byref(index), _ptr(scores),
         _ptr(list_partials), _ptr(sel_idx), _ptr(sel_count), _ptr(seq_lens), _ptr(out), _ptr(lse),
-        _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+        _ptr(out_f32), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def decode(params, q, index: Index, kv: PagedKV, seq_lens, out, ws, stream=None) -> None:
@@ -264,6 +275,15 @@ def decode_host(params, q_host, q_staging, index: Index, kv: PagedKV, seq_lens, 
         ctypes.byref(params), _ptr(q_host), _ptr(q_staging), ctypes.byref(index),
         ctypes.byref(kv), _ptr(seq_lens), _ptr(out_staging), _ptr(out_host), _ptr(ws),
         ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def debug_build() -> bool:
+    """True if the loaded library was built with -DPQHSA_DEBUG."""
+    return bool(lib().pqhsa_debug_build())
+
+
+def debug_predicate(which: int, value: int, lo: int, hi: int) -> int:
+    return lib().pqhsa_debug_predicate(which, value, lo, hi)
 
 
 def last_device_status(params, ws, stream=None) -> int:

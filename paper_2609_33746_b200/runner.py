@@ -13,7 +13,7 @@ class DecodeOp:
     """Device buffers + marshalled structs of one workload; every method is one library call."""
 
     def __init__(self, inp: DecodeInputs, index: IvfPqIndex, device: str = "cuda:0",
-                 budget_ppm: int | None = None):
+                 budget_ppm: int | None = None, variant: str | None = None):
         cfg: DecodeConfig = inp.cfg
         self.cfg, self.device = cfg, torch.device(device)
         dev = self.device
@@ -35,6 +35,10 @@ class DecodeOp:
         self.centroids, self.codebooks = put(index.centroids), put(index.codebooks)
         self.codes, self.list_ids = put(index.codes), put(index.list_ids)
         self.key_norms, self.list_vmeans = put(index.key_norms), put(index.list_vmeans)
+        self.list_counts = put(index.list_counts) if index.list_counts is not None else None
+        self.indexed_lens = None
+        if cfg.indexed_lens is not None:
+            self.indexed_lens = put(torch.tensor(list(cfg.indexed_lens), dtype=torch.int32))
 
         ppm = cfg.budget_ppm if budget_ppm is None else budget_ppm
         self.params = pqhsa.make_params(
@@ -42,9 +46,10 @@ class DecodeOp:
             n_list=cfg.n_list, pq_m=cfg.pq_m, max_seq_len=self.codes.shape[2],
             max_pages_per_seq=inp.max_pages_per_seq, budget_ppm=ppm, dtype=cfg.dtype,
             head_dim=cfg.head_dim, pq_ncode=cfg.pq_ncode, page_size=cfg.page_size, n_sink=cfg.n_sink,
-            n_local=cfg.n_local, exact_set_multiple=cfg.exact_set_multiple)
+            n_local=cfg.n_local, exact_set_multiple=cfg.exact_set_multiple,
+            variant=cfg.variant if variant is None else variant, indexed_lens=self.indexed_lens)
         self.index = pqhsa.make_index(self.centroids, self.codebooks, self.codes, self.list_ids,
-                                      self.key_norms, self.list_vmeans)
+                                      self.key_norms, self.list_vmeans, self.list_counts)
         self.kv = pqhsa.make_paged_kv(self.k_cache, self.v_cache, inp.stride_page,
                                       inp.stride_token, inp.stride_head, self.block_table)
         self.ws = torch.empty(pqhsa.workspace_bytes(self.params), dtype=torch.uint8, device=dev)
@@ -63,6 +68,7 @@ class DecodeOp:
         self.sel_idx, self.sel_count = i32(pqhsa.BUF_SEL_IDX), i32(pqhsa.BUF_SEL_COUNT)
         self.kth = f32(pqhsa.BUF_KTH)
         self.lse = torch.empty(p.batch * p.n_q_heads, dtype=torch.float32, device=dev)
+        self.out_f32 = torch.empty(self.q.shape, dtype=torch.float32, device=dev)
 
     def build_lut(self):
         pqhsa.build_lut(self.params, self.q, self.index, self.lut, self.coarse)
@@ -78,7 +84,7 @@ class DecodeOp:
     def hybrid_attend(self):
         pqhsa.hybrid_attend(self.params, self.q, self.kv, self.index, self.scores,
                             self.list_partials, self.sel_idx, self.sel_count, self.seq_lens,
-                            self.out, self.lse, self.ws)
+                            self.out, self.lse, self.ws, out_f32=self.out_f32)
 
     def decode(self, q=None, out=None):
         pqhsa.decode(self.params, self.q if q is None else q, self.index, self.kv, self.seq_lens,

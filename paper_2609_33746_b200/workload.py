@@ -55,6 +55,9 @@ class DecodeConfig:
     n_sink: int = 0                      # |S|: first tokens attended exactly (Sec. 3.2)
     n_local: int = 0                     # |L|: most recent tokens attended exactly
     exact_set_multiple: int = 0          # >1: |S|+|L|+k rounded up to this multiple (App. A)
+    variant: str = "B"                   # background term: B (PQ-HSA), T, Bx, C, C2, C2b (Table 2)
+    indexed_lens: Optional[tuple] = None # per sequence: positions the index covers; the rest of
+                                         # the sequence is the exactly-attended window (Sec. 3.3)
 
     @property
     def group(self) -> int:

@@ -64,7 +64,8 @@ def oracle_arrays_for_sequence(inp, idx, b):
         seq_lens=inp.seq_lens[sl].cpu().numpy())
 
 
-def run_oracle(inp, idx, budget_ppm=None, heads=None, batch_items=None, arrays=None):
+def run_oracle(inp, idx, budget_ppm=None, heads=None, batch_items=None, arrays=None, variant=None,
+               indexed_lens=None):
     cfg = inp.cfg
     a = arrays or oracle_arrays(inp, idx)
     return O.decode(a["q"], a["centroids"], a["codebooks"], a["codes"], a["list_ids"],
@@ -75,6 +76,8 @@ def run_oracle(inp, idx, budget_ppm=None, heads=None, batch_items=None, arrays=N
                     budget_ppm=cfg.budget_ppm if budget_ppm is None else budget_ppm,
                     sm_scale=1.0 / math.sqrt(cfg.head_dim), heads=heads, batch_items=batch_items,
                     n_sink=cfg.n_sink, n_local=cfg.n_local,
+                    variant=cfg.variant if variant is None else variant,
+                    indexed_lens=cfg.indexed_lens if indexed_lens is None else indexed_lens,
                     round_exact_set_to_page=cfg.exact_set_multiple if cfg.exact_set_multiple > 1 else 0)
 
 

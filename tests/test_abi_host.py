@@ -95,3 +95,14 @@ def test_status_strings():
     assert pqhsa.status_string(0) == "ok"
     assert "workspace" in pqhsa.status_string(pqhsa.ERR_WORKSPACE)
     assert pqhsa.status_string(-99) == "unknown status"
+
+
+def test_debug_check_predicates_on_the_host():
+    """The predicates behind the -DPQHSA_DEBUG index checks (list id, selected position, page id),
+    exercised on the host: the GPU is never fed a bad index on purpose."""
+    P = pqhsa.debug_predicate
+    assert [P(0, v, 0, 64) for v in (0, 63, 64, 65535, -1)] == [1, 1, 0, 0, 0]          # list id < n_list
+    assert [P(1, v, 4, 100) for v in (3, 4, 99, 100, -7)] == [0, 1, 1, 0, 0]            # r_begin <= pos < r_end
+    assert [P(2, v, 0, 0) for v in (0, 12345, -1)] == [1, 1, 0]                         # page id >= 0
+    assert P(9, 0, 0, 0) == -1
+    assert pqhsa.debug_build() in (False, True)

@@ -4,12 +4,17 @@
 // One pass over the scores instead of a multi-pass radix sort of the whole row:
 //   sample kernel  one CTA per row reads 4096 scores (1024 groups of 4, jittered stride)
 //                  and takes two order statistics of the sample that bracket the k-th largest
-//                  score of the row with a 6-sigma margin: lo <= s_k <= hi;
+//                  score of the row with a 6-sigma margin: lo <= s_k <= hi (one histogram of
+//                  the sample over 4096 equal buckets of its range; the bracket's edges are
+//                  bucket edges);
 //   filter kernel  scores above hi are certain winners and are written out at once; scores in
 //                  [lo, hi] (a few percent of k) are appended to a candidate list; the last
 //                  CTA of the row (atomic ticket, nobody waits) checks the bracket by counting
-//                  (#winners <= k <= #winners + #candidates) and finishes with an exact
-//                  12/12/8-bit radix select over the candidates.
+//                  (#winners <= k <= #winners + #candidates) and finishes exactly: one
+//                  histogram of the candidates over 4096 equal buckets of [lo, hi], everything
+//                  above the bucket of the k-th largest is taken, the few items inside it are
+//                  ranked against each other (a 12/12/8-bit radix select remains for candidate
+//                  sets that do not fit shared memory or pile up in one bucket).
 // If the bracket misses (a row whose order defeats the sample), that last CTA redoes the
 // row from the scores themselves with the same radix select, so the result is always the
 // exact top-k; equal scores at the threshold are taken in order of position (lowest first),
@@ -141,37 +146,57 @@ __device__ __forceinline__ void load_chunk(const float* __restrict__ rs, int chu
 }
 
 // ------------------------------------------------------------------------- sample kernel
-// 24-bit prefixes (key >> 8) of the rank_a-th and rank_b-th largest (0-based) of the CTA's 4096
-// sampled keys (8 per thread, in registers).  Two 12-bit digits; both ranks share each pass.
-__device__ void sample_prefixes(const uint32_t (&key)[kSamplePer], int rank_a, int rank_b,
-                                uint32_t* s_hist, uint32_t* s_hist_b, int* s_scan,
-                                uint32_t& pre_a, uint32_t& pre_b) {
-  const int tid = threadIdx.x;
-  int d, above;
-  for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
-  __syncthreads();
+// Bucket of a score in a linear partition of [lo, lo + kHistBins / scale) into kHistBins
+// buckets; a larger score never gets a smaller bucket (the product is monotone and clamped).
+__device__ __forceinline__ int linear_bucket(float s, float lo, float scale) {
+  const float t = (s - lo) * scale;
+  return t >= (float)(kHistBins - 1) ? kHistBins - 1 : (t > 0.f ? (int)t : 0);   // NaN -> 0
+}
+
+// Buckets (from the top) that hold the rank_a-th and rank_b-th largest (0-based) of the items
+// counted in `hist`; one pass over the histogram serves both ranks.
+__device__ void find_two_buckets(const uint32_t* hist, int rank_a, int rank_b, int* s_scan,
+                                 int& bucket_a, int& bucket_b) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int per = kHistBins / kSelThreads;                 // 8 bins per thread, top down
+  const int hi = kHistBins - tid * per;
+  const uint4 v0 = *reinterpret_cast<const uint4*>(hist + hi - 8);
+  const uint4 v1 = *reinterpret_cast<const uint4*>(hist + hi - 4);
+  const uint32_t mine[8] = {v1.w, v1.z, v1.y, v1.x, v0.w, v0.z, v0.y, v0.x};
+  uint32_t local = 0;
 #pragma unroll
-  for (int e = 0; e < kSamplePer; ++e) atomicAdd(&s_hist[key[e] >> 20], 1u);
-  __syncthreads();
-  find_digit(s_hist, kHistBins, rank_a + 1, s_scan, d, above);
-  const uint32_t a1 = (uint32_t)d;
-  const int need_a = rank_a + 1 - above;
-  find_digit(s_hist, kHistBins, rank_b + 1, s_scan, d, above);
-  const uint32_t b1 = (uint32_t)d;
-  const int need_b = rank_b + 1 - above;
-  for (int i = tid; i < kHistBins; i += kSelThreads) { s_hist[i] = 0u; s_hist_b[i] = 0u; }
-  __syncthreads();
+  for (int j = 0; j < 8; ++j) local += mine[j];
+  if (tid == 0) { s_scan[32] = 0; s_scan[33] = 0; }
+  uint32_t inc = local;
 #pragma unroll
-  for (int e = 0; e < kSamplePer; ++e) {
-    const uint32_t t = key[e] >> 20, lo12 = (key[e] >> 8) & 0xfffu;
-    if (t == a1) atomicAdd(&s_hist[lo12], 1u);
-    if (t == b1) atomicAdd(&s_hist_b[lo12], 1u);
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += v;
+  }
+  if (lane == 31) s_scan[warp] = (int)inc;
+  __syncthreads();
+  if (warp == 0) {
+    const int v = (lane < kSelThreads / 32) ? s_scan[lane] : 0;
+    int w = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += u;
+    }
+    if (lane < kSelThreads / 32) s_scan[lane] = w - v;       // exclusive warp offsets
   }
   __syncthreads();
-  find_digit(s_hist, kHistBins, need_a, s_scan, d, above);
-  pre_a = (a1 << 12) | (uint32_t)d;
-  find_digit(s_hist_b, kHistBins, need_b, s_scan, d, above);
-  pre_b = (b1 << 12) | (uint32_t)d;
+  uint32_t run = (uint32_t)s_scan[warp] + inc - local;       // items in buckets above mine
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    if (run <= (uint32_t)rank_a && (uint32_t)rank_a < run + mine[j]) s_scan[32] = hi - 1 - j;
+    if (run <= (uint32_t)rank_b && (uint32_t)rank_b < run + mine[j]) s_scan[33] = hi - 1 - j;
+    run += mine[j];
+  }
+  __syncthreads();
+  bucket_a = s_scan[32];
+  bucket_b = s_scan[33];
+  __syncthreads();
 }
 
 __global__ void __launch_bounds__(kSelThreads)
@@ -179,9 +204,9 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
                   int32_t* __restrict__ rowstate, int32_t* __restrict__ sel_count,
                   float* __restrict__ kth) {
   __shared__ __align__(16) uint32_t s_hist[kHistBins];
-  __shared__ __align__(16) uint32_t s_hist_b[kHistBins];
   __shared__ int s_scan[34];
-  const int row = blockIdx.x, tid = threadIdx.x;
+  __shared__ float s_mm[2][kSelThreads / 32];
+  const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = row / pl.Hq;
   pdl_wait();
   pdl_launch_dependents();
@@ -208,23 +233,49 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
       const float4 f = __ldcg(reinterpret_cast<const float4*>(rs + off));
       s[4 * u] = f.x; s[4 * u + 1] = f.y; s[4 * u + 2] = f.z; s[4 * u + 3] = f.w;
     }
-    uint32_t key[kSamplePer];
+    for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;   // while the loads fly
+    // range of the finite samples (sink and window positions hold -inf)
+    float mn = CUDART_INF_F, mx = -CUDART_INF_F;
 #pragma unroll
-    for (int e = 0; e < kSamplePer; ++e) key[e] = score_key(s[e]);
+    for (int e = 0; e < kSamplePer; ++e) {
+      const bool fin = fabsf(s[e]) < CUDART_INF_F;
+      mn = fin ? fminf(mn, s[e]) : mn;
+      mx = fin ? fmaxf(mx, s[e]) : mx;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    if (lane == 0) { s_mm[0][warp] = mn; s_mm[1][warp] = mx; }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kSelThreads / 32; ++w) { mn = fminf(mn, s_mm[0][w]); mx = fmaxf(mx, s_mm[1][w]); }
     // the k-th largest of the row sits near rank p*4096 of the sample; the bracket is
     // +- 6 sigma of that count (binomial bound on the hypergeometric spread), + 2
     const float p = (float)k / (float)n;
     const float r = p * kSample;
     const int mgn = (int)ceilf(kBracketSigmas * sqrtf(kSample * p * (1.f - p))) + 2;
     const int r_hi = (int)floorf(r) - mgn, r_lo = (int)ceilf(r) + mgn;
-    // the bracket only has to contain the two order statistics: take the edges of their
-    // 24-bit key prefixes (256 ulps wide), which saves the third radix digit
-    uint32_t pre_hi, pre_lo;
-    sample_prefixes(key, max(r_hi, 0), min(r_lo, kSample - 1), s_hist, s_hist_b, s_scan, pre_hi,
-                    pre_lo);
-    if (r_hi >= 0) hi = key_score((pre_hi << 8) | 0xffu);
-    if (r_lo < kSample) lo = key_score(pre_lo << 8);
-    if (hi != hi) hi = CUDART_INF_F;                 // prefix that runs into the NaN patterns
+    if (mx > mn) {
+      // one histogram of the samples over 4096 equal buckets of [mn, mx] (non-finite samples
+      // fall into the bottom bucket); the bracket is the outer edges of the two buckets that
+      // hold the order statistics, one bucket wider on each side for the rounding of the edges.
+      // Whatever the bracket is, the filter kernel checks it by counting.
+      const float scale = (float)kHistBins / (mx - mn);
+#pragma unroll
+      for (int e = 0; e < kSamplePer; ++e) atomicAdd(&s_hist[linear_bucket(s[e], mn, scale)], 1u);
+      __syncthreads();
+      int b_hi, b_lo;
+      find_two_buckets(s_hist, max(r_hi, 0), min(r_lo, kSample - 1), s_scan, b_hi, b_lo);
+      const float width = (mx - mn) / (float)kHistBins;
+      if (r_hi >= 0) hi = mn + (float)(b_hi + 2) * width;
+      if (r_lo < kSample && b_lo >= 2) lo = mn + (float)(b_lo - 1) * width;
+    } else if (mx == mn) {
+      hi = mx;                                     // all finite samples equal: take that value
+      lo = mn;                                     // as the whole bracket
+    }
+    if (hi != hi) hi = CUDART_INF_F;
     if (lo != lo) lo = -CUDART_INF_F;
   }
   if (tid == 0) {
@@ -368,7 +419,7 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
   uint32_t* s_hits = reinterpret_cast<uint32_t*>(s_raw);          // [16 warps][512]
   __shared__ int s_scan[34];
   __shared__ int s_last;
-  __shared__ uint32_t s_emit;
+  __shared__ uint32_t s_emit, s_tie, s_kstar;
   const int row = blockIdx.y, tid = threadIdx.x, chunk = blockIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   pdl_wait();
@@ -513,8 +564,58 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
         __syncthreads();
         src = kFromStash;
       }
-      kstar = resolve_top_r(src, s_stash, rc, C, rs, n, r, out, (uint32_t)W, pl.k_max, s_hist,
-                            s_scan, &s_emit);
+      bool done = false;
+      if (src == kFromStash && lo_f > -CUDART_INF_F && hi_f < CUDART_INF_F && hi_f > lo_f) {
+        // Fast finish.  The staged candidates all lie in [lo, hi]: ONE histogram over 4096
+        // equal buckets of that interval finds the bucket of the r-th largest; everything in a
+        // higher bucket is taken at once, and the few items of that bucket are ranked against
+        // each other (larger score first, then lower position: the stable rule).
+        const float scale = (float)kHistBins / (hi_f - lo_f);
+        for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
+        __syncthreads();
+        for (int i = tid; i < C; i += kSelThreads)
+          atomicAdd(&s_hist[linear_bucket(key_score(s_stash[i].x), lo_f, scale)], 1u);
+        __syncthreads();
+        int d, above;
+        find_digit(s_hist, kHistBins, r, s_scan, d, above);
+        const int m = (int)s_hist[d], need = r - above;        // 1 <= need <= m
+        __syncthreads();                                         // everybody has read s_hist[d]
+        constexpr int kTieCap = kHistBins / 2;                   // (key, position) pairs in s_hist's place
+        if (m <= kTieCap) {
+          uint2* tie = reinterpret_cast<uint2*>(s_hist);
+          if (tid == 0) s_tie = 0u;
+          __syncthreads();
+          for (int base = 0; base < C; base += kSelThreads) {
+            const int i = base + tid;
+            const bool v = i < C;
+            const uint2 it = v ? s_stash[i] : make_uint2(0u, 0u);
+            const int bk = v ? linear_bucket(key_score(it.x), lo_f, scale) : -1;
+            const int p = warp_append(v && bk > d, &s_emit);
+            if (p >= 0 && (uint32_t)W + p < (uint32_t)pl.k_max) out[W + p] = (int)it.y;
+            if (v && bk == d) tie[atomicAdd(&s_tie, 1u)] = it;
+          }
+          __syncthreads();
+          for (int base = 0; base < m; base += kSelThreads) {
+            const int i = base + tid;
+            const bool v = i < m;
+            const uint2 me = v ? tie[i] : make_uint2(0u, 0u);
+            int rank = 0;
+            for (int j = 0; j < m; ++j) {
+              const uint2 o = tie[j];
+              rank += (o.x > me.x || (o.x == me.x && o.y < me.y)) ? 1 : 0;
+            }
+            const int p = warp_append(v && rank < need, &s_emit);
+            if (p >= 0 && (uint32_t)W + p < (uint32_t)pl.k_max) out[W + p] = (int)me.y;
+            if (v && rank == need - 1) s_kstar = me.x;
+          }
+          __syncthreads();
+          kstar = s_kstar;
+          done = true;
+        }
+      }
+      if (!done)
+        kstar = resolve_top_r(src, s_stash, rc, C, rs, n, r, out, (uint32_t)W, pl.k_max, s_hist,
+                              s_scan, &s_emit);
     }
   } else {
     // the sample's bracket missed: redo the row from the scores (slow, exact)

@@ -267,6 +267,34 @@ int pqhsa_index_update(const pqhsa_params* params, const pqhsa_index_rw* index,
                        const pqhsa_paged_kv* kv, const int32_t* first_pos, const int32_t* n_new,
                        int32_t max_new, void* stream);
 
+/* Batched index build (Sec. 3.3, first paragraph; App. C, "Index build"): trains the IVF-PQ
+ * index of EVERY (sequence, KV head) in one call, one launch per step for all of them, from the
+ * keys and values in the paged cache.  Per unit: r_i = |k_i| (fp32), u_i = k_i / r_i (0 for a
+ * zero key); `coarse_iters` Lloyd iterations on the directions from the centroids seeded with the
+ * tokens at seed_lists[b][kv][j] (squared Euclidean distance, lower index on ties, centroid =
+ * arithmetic mean of its members, an empty list is re-seeded with the farthest point; a negative
+ * seed position gives a zero row), then the final assignment a_i; `pq_iters` Lloyd iterations per
+ * subspace on the residuals u_i - c_{a_i} from the codewords seeded with the residuals of the
+ * tokens at seed_codes[b][kv][z], then the final codes; the list value means over the members
+ * inside R_b and the member counts.  The two seed arrays are the method's random draws: device
+ * int32 [B][H_kv][n_list] and [B][H_kv][pq_ncode].  All arrays of `index` are outputs.
+ * ws: pqhsa_index_build_workspace_bytes(params) bytes (it holds the fp32 directions: 512 bytes
+ * per token and KV head), 256-byte aligned.  Launches only; no synchronisation. */
+typedef struct {
+  float* centroids;           /* [B][H_kv][n_list][d]                                        */
+  float* codebooks;           /* [B][H_kv][M][pq_ncode][dsub]                                */
+  uint8_t* codes;             /* [B][H_kv][N_max][M] (or [M/2] with pq_ncode == 16)          */
+  uint16_t* list_ids;         /* [B][H_kv][N_max]                                            */
+  float* key_norms;           /* [B][H_kv][N_max]                                            */
+  float* list_vmeans;         /* [B][H_kv][n_list][d]                                        */
+  int32_t* list_counts;       /* [B][H_kv][n_list]                                           */
+} pqhsa_index_out;
+size_t pqhsa_index_build_workspace_bytes(const pqhsa_params* params);
+int pqhsa_index_build(const pqhsa_params* params, const pqhsa_paged_kv* kv, const int32_t* seq_lens,
+                      const int32_t* seed_lists, const int32_t* seed_codes, int32_t coarse_iters,
+                      int32_t pq_iters, const pqhsa_index_out* index, void* ws, size_t ws_bytes,
+                      void* stream);
+
 /* Dense decode attention over the WHOLE paged KV cache (Eq. 1 with E = every cached token):
  * softmax(q K^T / sqrt d) V per query head, split-K with a log-sum-exp merge.  Not a step of
  * PQ-HSA: it is the comparator of the context-length sweep (the full-KV read the paper's

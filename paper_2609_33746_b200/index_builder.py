@@ -133,8 +133,7 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
         if n == 0:
             continue
         for g in range(Hkv):
-            gen = torch.Generator(device=dev).manual_seed(
-                (cfg.seed * 1000003 + b * 4099 + g * 17 + 7) & 0x7FFFFFFF)
+            gen = torch.Generator(device=dev).manual_seed(_unit_seed(cfg, b, g))
             k, v = inp.gather_kv(b, g)
             k32 = k.float()
             r = k32.norm(dim=1)                                   # fp32 norms
@@ -146,7 +145,8 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
             c = _kmeans(fit, nl, cfg.kmeans_iters, gen)
             ids, _ = _assign(u, c)
             res_fit = (fit - c[_assign(fit, c)[0]]) if fit is not u else (u - c[ids])
-            cb = _batched_pq_kmeans(res_fit.view(-1, M, dsub), nc, cfg.kmeans_iters, gen)
+            cb = _batched_pq_kmeans(res_fit.view(-1, M, dsub), nc,
+                                    cfg.kmeans_iters if cfg.pq_iters is None else cfg.pq_iters, gen)
             res = (u - c[ids]).view(n, M, dsub).permute(1, 0, 2).contiguous()
             codes = _pq_encode(res, cb)                           # [M, n]
             # list value means over the members inside the indexed region R (Sec. 3.2): sink
@@ -169,4 +169,79 @@ def build_index(inp: DecodeInputs) -> IvfPqIndex:
             out.key_norms[b, g, :n] = r
             out.list_vmeans[b, g] = vmean.float()
             out.list_counts[b, g] = cnt.to(torch.int32)
+    return out
+
+
+def _unit_seed(cfg: DecodeConfig, b: int, g: int) -> int:
+    return (cfg.seed * 1000003 + b * 4099 + g * 17 + 7) & 0x7FFFFFFF
+
+
+def seed_positions(inp: DecodeInputs):
+    """The random draws of build_index, on their own: for every (sequence, KV head) the
+    positions of the tokens that seed the centroids [B, Hkv, n_list] and the codewords
+    [B, Hkv, pq_ncode] (-1 where the sequence has fewer tokens than seeds).  Same generator,
+    same order of draws as build_index (without fit_sample), so that another builder started
+    from these positions trains the same problems."""
+    cfg = inp.cfg
+    dev = inp.q.device
+    lists = torch.full((cfg.batch, cfg.n_kv_heads, cfg.n_list), -1, dtype=torch.int32, device=dev)
+    words = torch.full((cfg.batch, cfg.n_kv_heads, cfg.pq_ncode), -1, dtype=torch.int32, device=dev)
+    for b in range(cfg.batch):
+        n = cfg.seq_lens[b]
+        if n == 0:
+            continue
+        for g in range(cfg.n_kv_heads):
+            gen = torch.Generator(device=dev).manual_seed(_unit_seed(cfg, b, g))
+            if n >= cfg.n_list:
+                lists[b, g] = torch.randperm(n, generator=gen, device=dev)[:cfg.n_list].int()
+            else:
+                lists[b, g, :n] = torch.arange(n, dtype=torch.int32, device=dev)
+            if n >= cfg.pq_ncode:
+                words[b, g] = torch.randperm(n, generator=gen, device=dev)[:cfg.pq_ncode].int()
+            else:
+                words[b, g, :n] = torch.arange(n, dtype=torch.int32, device=dev)
+    return lists, words
+
+
+def build_index_batched(inp: DecodeInputs, coarse_iters=None, pq_iters=None) -> IvfPqIndex:
+    """The index of a workload trained by the library's batched build (pqhsa_index_build): all
+    (sequence, KV head) problems in one call, from the same seed positions as build_index."""
+    from . import pqhsa
+    cfg = inp.cfg
+    dev = inp.q.device
+    B, Hkv, d = cfg.batch, cfg.n_kv_heads, cfg.head_dim
+    M, dsub, nl, nc = cfg.pq_m, cfg.pq_dsub, cfg.n_list, cfg.pq_ncode
+    Nmax = max(16, (cfg.max_seq_len + 15) // 16 * 16)
+    out = IvfPqIndex(
+        torch.zeros((B, Hkv, nl, d), dtype=torch.float32, device=dev),
+        torch.zeros((B, Hkv, M, nc, dsub), dtype=torch.float32, device=dev),
+        torch.zeros((B, Hkv, Nmax, M if nc > 16 else M // 2), dtype=torch.uint8, device=dev),
+        torch.zeros((B, Hkv, Nmax), dtype=torch.int16, device=dev),
+        torch.zeros((B, Hkv, Nmax), dtype=torch.float32, device=dev),
+        torch.zeros((B, Hkv, nl, d), dtype=torch.float32, device=dev),
+        torch.zeros((B, Hkv, nl), dtype=torch.int32, device=dev))
+    indexed = None
+    if cfg.indexed_lens is not None:
+        indexed = torch.tensor(list(cfg.indexed_lens), dtype=torch.int32, device=dev)
+    params = pqhsa.make_params(
+        batch=B, n_q_heads=cfg.n_q_heads, n_kv_heads=Hkv, n_list=nl, pq_m=M, max_seq_len=Nmax,
+        max_pages_per_seq=inp.max_pages_per_seq, budget_ppm=cfg.budget_ppm, dtype=cfg.dtype,
+        head_dim=d, pq_ncode=nc, page_size=cfg.page_size, n_sink=cfg.n_sink, n_local=cfg.n_local,
+        exact_set_multiple=cfg.exact_set_multiple, indexed_lens=indexed)
+    if cfg.kv_layout == "interleaved":
+        k_cache, v_cache = inp.k_cache, inp.k_cache.view(-1)[d:]
+    else:
+        k_cache, v_cache = inp.k_cache, inp.v_cache
+    kv = pqhsa.make_paged_kv(k_cache, v_cache, inp.stride_page, inp.stride_token, inp.stride_head,
+                             inp.block_table)
+    lists, words = seed_positions(inp)
+    ws = torch.empty(pqhsa.index_build_workspace_bytes(params), dtype=torch.uint8, device=dev)
+    it = cfg.kmeans_iters
+    it_pq = it if cfg.pq_iters is None else cfg.pq_iters
+    pqhsa.index_build(params, kv, inp.seq_lens, lists, words,
+                      it if coarse_iters is None else coarse_iters,
+                      it_pq if pq_iters is None else pq_iters,
+                      out.centroids, out.codebooks, out.codes, out.list_ids, out.key_norms,
+                      out.list_vmeans, out.list_counts, ws)
+    torch.cuda.synchronize(dev)
     return out

@@ -31,7 +31,7 @@ EXPORTS = [
     "pqhsa_decode_launch_count", "pqhsa_status_string", "pqhsa_select_static",
     "pqhsa_select_static_bytes", "pqhsa_select_static_capacity", "pqhsa_dense_decode",
     "pqhsa_dense_workspace_bytes", "pqhsa_index_update", "pqhsa_debug_build",
-    "pqhsa_debug_predicate",
+    "pqhsa_debug_predicate", "pqhsa_index_build", "pqhsa_index_build_workspace_bytes",
 ]
 
 
@@ -56,6 +56,11 @@ class Index(ctypes.Structure):
 
 
 class IndexRW(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in (
+        "centroids", "codebooks", "codes", "list_ids", "key_norms", "list_vmeans", "list_counts")]
+
+
+class IndexOut(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in (
         "centroids", "codebooks", "codes", "list_ids", "key_norms", "list_vmeans", "list_counts")]
 
@@ -101,6 +106,8 @@ def lib() -> ctypes.CDLL:
             "pqhsa_dense_decode": (I, [P, V, PK, V, V, V, Z, V]),
             "pqhsa_dense_workspace_bytes": (Z, [P]),
             "pqhsa_index_update": (I, [P, ctypes.POINTER(IndexRW), PK, V, V, I, V]),
+            "pqhsa_index_build_workspace_bytes": (Z, [P]),
+            "pqhsa_index_build": (I, [P, PK, V, V, V, I, I, ctypes.POINTER(IndexOut), V, Z, V]),
             "pqhsa_debug_build": (I, []),
             "pqhsa_debug_predicate": (I, [I, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_longlong]),
         }
@@ -274,6 +281,24 @@ def decode_host(params, q_host, q_staging, index: Index, kv: PagedKV, seq_lens, 
     _check("pqhsa_decode_host", lib().pqhsa_decode_host(
         ctypes.byref(params), _ptr(q_host), _ptr(q_staging), ctypes.byref(index),
         ctypes.byref(kv), _ptr(seq_lens), _ptr(out_staging), _ptr(out_host), _ptr(ws),
+        ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def index_build_workspace_bytes(params: Params) -> int:
+    return lib().pqhsa_index_build_workspace_bytes(ctypes.byref(params))
+
+
+def index_build(params, kv: PagedKV, seq_lens, seed_lists, seed_codes, coarse_iters: int, pq_iters: int,
+                centroids, codebooks, codes, list_ids, key_norms, list_vmeans, list_counts, ws,
+                stream=None) -> None:
+    """Trains the index of every (sequence, KV head) at once from the paged cache; every index
+    tensor is an output.  seed_lists / seed_codes: the positions whose tokens seed the centroids
+    and the codewords (the method's random draws)."""
+    out = IndexOut(_ptr(centroids), _ptr(codebooks), _ptr(codes), _ptr(list_ids), _ptr(key_norms),
+                   _ptr(list_vmeans), _ptr(list_counts))
+    _check("pqhsa_index_build", lib().pqhsa_index_build(
+        ctypes.byref(params), ctypes.byref(kv), _ptr(seq_lens), _ptr(seed_lists), _ptr(seed_codes),
+        int(coarse_iters), int(pq_iters), ctypes.byref(out), _ptr(ws),
         ws.numel() * ws.element_size(), _stream(stream)))
 
 

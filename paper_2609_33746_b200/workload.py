@@ -48,6 +48,7 @@ class DecodeConfig:
     page_size: int = PAGE_SIZE
     outlier_scale: float = 8.0
     kmeans_iters: int = 10
+    pq_iters: Optional[int] = None       # Lloyd iterations of the codebooks (None: kmeans_iters)
     seed: int = 0
     kv_layout: str = "split"             # "split": K and V separate [page][tok][head][d]
                                          # "interleaved": one buffer [page][head][tok][2d]

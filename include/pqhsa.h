@@ -228,7 +228,8 @@ int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_p
  *     is launched; use pqhsa_select with your own workspace for those.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current).  Make that first call outside any
- *     stream capture.
+ *     stream capture.  The address is kept per device for the life of the process: after a
+ *     cudaDeviceReset the library has to be loaded again before this entry point is used.
  *   - All calls on a device share the one array and it keeps the last call's contents; each
  *     call clears the part that must start at zero on `stream` first.  Two calls that can
  *     overlap on the GPU (different streams, no dependency) race on it: serialise them.

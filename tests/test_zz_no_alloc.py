@@ -58,6 +58,12 @@ def test_select_static_matches_select_on_two_calls_in_a_row():
         pqhsa.select_static(op.params, op.scores, op.seq_lens, op.sel_idx, op.sel_count, op.kth)
         torch.cuda.synchronize()
         got_sets, got_cnt, got_kth = _sets(op, cfg)
+        # what the entry point is for: a call allocates nothing (the driver's count of free
+        # device memory is the same before and after a repeat of the call)
+        free_before = torch.cuda.mem_get_info()[0]
+        pqhsa.select_static(op.params, op.scores, op.seq_lens, op.sel_idx, op.sel_count, op.kth)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
         assert np.array_equal(got_cnt, want_cnt), f"call {call}: counts differ"
         # the selection is exact and tie-stable in both entry points: identical sets
         assert got_sets == want_sets, f"call {call}: selected sets differ"

@@ -80,6 +80,8 @@ typedef struct {
                               /* k_max must then cover the extra m - 1                        */
   int32_t variant;            /* pqhsa_variant: how the background term is formed (Table 2);  */
                               /* 0 = PQ-HSA itself                                            */
+  int32_t table_precision;    /* pqhsa_table_precision: 0 = fp32 lookup tables (the mode every  */
+                              /* stated tolerance refers to), 1 = fp16 tables in the scan        */
   const int32_t* indexed_lens;/* DEVICE pointer [B] or NULL.  Number of leading positions of  */
                               /* each sequence that the index covers: R_b = [|S_b|,           */
                               /* indexed_lens[b]) and L_b = everything after (Sec. 3.3: a new */
@@ -87,6 +89,16 @@ typedef struct {
                               /* encodes it).  NULL: L_b is the last n_local tokens.  Values  */
                               /* are clipped to [|S_b|, seq_lens[b]]; n_local is then unused  */
 } pqhsa_params;
+
+/* Precision of the scan's lookup tables.  PQHSA_TABLES_FP16 is an opt-in fast mode (in the spirit of
+ * Sec. 1 / Sec. 6: the scan is an IVF-PQ scan and takes that literature's reduced-precision tables):
+ * the table build is unchanged, the scan holds the tables as fp16 and sums four entries in fp16
+ * before it widens them, so an approximate logit carries an error of about 1e-3 of the table
+ * entries' magnitude instead of fp32 rounding.  Everything downstream is unchanged: the top-k is
+ * exact on those scores, the selected tokens are attended with exact logits, and the list sums use
+ * the same approximate logits that are later taken out of them.  v1: pq_ncode == 256, pq_m == 32,
+ * G >= 3 (groups of four heads). */
+typedef enum { PQHSA_TABLES_FP32 = 0, PQHSA_TABLES_FP16 = 1 } pqhsa_table_precision;
 
 /* Mechanism variants of the paper's ablation (Table 2; App. B, "Variant definitions").  All of
  * them keep the selector, the budget and the exact part; they differ in the background term.

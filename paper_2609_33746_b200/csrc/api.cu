@@ -50,6 +50,8 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (p->dtype != PQHSA_F16 && p->dtype != PQHSA_BF16) return PQHSA_ERR_INVALID_ARG;
   if (!(p->sm_scale > 0.f)) return PQHSA_ERR_INVALID_ARG;
   if (p->variant < PQHSA_VARIANT_B || p->variant > PQHSA_VARIANT_C2B) return PQHSA_ERR_INVALID_ARG;
+  if (p->table_precision != PQHSA_TABLES_FP32 && p->table_precision != PQHSA_TABLES_FP16)
+    return PQHSA_ERR_INVALID_ARG;
   if ((long long)p->max_pages_per_seq * p->page_size < p->max_seq_len) return PQHSA_ERR_INVALID_ARG;
   long long k_need = ((long long)p->max_seq_len * p->budget_ppm + 999999LL) / 1000000LL;
   if (p->exact_set_multiple > 1) k_need += p->exact_set_multiple - 1;     // rounding slack
@@ -67,6 +69,9 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (p->n_list > 4096 || p->max_seq_len % 4 != 0) return PQHSA_ERR_UNSUPPORTED;
   const int G = p->n_q_heads / p->n_kv_heads;
   if (G > 16) return PQHSA_ERR_UNSUPPORTED;
+  // fp16 tables: the layer shape of the benchmark only (32 one-byte subspaces, groups of 4 heads)
+  if (p->table_precision == PQHSA_TABLES_FP16 && (p->pq_ncode != 256 || p->pq_m != 32 || G < 3))
+    return PQHSA_ERR_UNSUPPORTED;
 
   Plan& o = *pl;
   o.B = p->batch; o.Hq = p->n_q_heads; o.Hkv = p->n_kv_heads; o.G = G;
@@ -78,6 +83,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.k_max = p->k_max; o.n_sink = p->n_sink; o.n_local = p->n_local;
   o.exact_multiple = p->exact_set_multiple; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
   o.variant = p->variant; o.indexed_lens = p->indexed_lens; o.status = nullptr;
+  o.half_tables = p->table_precision == PQHSA_TABLES_FP16 ? 1 : 0;
   o.num_sms = sm_count();
   o.scan_ctas = o.num_sms;                                  // persistent scan CTAs: one per SM
   o.upb = o.Hkv * o.n_hg;

@@ -35,6 +35,7 @@ struct Plan {
   int n_sink, n_local;               // |S| and |L| of Sec. 3.2 (upper bounds: clipped per sequence)
   int exact_multiple;                // > 1: |S| + |L| + k is rounded up to this multiple (App. A)
   int variant;                       // pqhsa_variant: how the background term is formed
+  int half_tables;                   // scan keeps its lookup tables in fp16 (approximate scores)
   const int32_t* indexed_lens;       // device [B] or null: positions covered by the index
   int* status;                       // device status word, or null (set by the launchers)
   uint32_t ppm;

@@ -117,7 +117,11 @@ __device__ __forceinline__ void read_codes(uint32_t slot, int lane, uint32_t (&w
 }
 
 // One byte per code, 256-entry tables (4-bit codes: scan4.cu).
-template <int M, int GC, int kStages>
+// kHalf (M = 32, GC = 4 only): the tables are held in shared memory as fp16 (8 bytes per entry
+// of four heads), which halves the table reads that bound the kernel.  The scores are then
+// approximate (about 1e-3 relative per table entry instead of 6e-8): an opt-in mode, not the one
+// the parity tolerances of the scan stage are stated for.
+template <int M, int GC, int kStages, bool kHalf>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restrict__ lids,
             const float* __restrict__ norms, const float* __restrict__ lut,
@@ -148,14 +152,22 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   const int c = blockIdx.x;
   const int n_list = pl.n_list, N_max = pl.N_max, upb = pl.upb;
 
-  pdl_wait();
+  // The tables come from the kernel right before this one (the table build); everything else
+  // this kernel reads is an input of the call, and what it writes (scores, list partials) is
+  // read only by later kernels.  Every CTA of the table build waits for ITS predecessors before
+  // it releases this grid, so a CTA of this kernel may run ahead of its own dependency wait
+  // until it needs the tables: the split, the first code copies, the first token metadata and
+  // the clearing of its partial overlap the tail of the table build.
   pdl_launch_dependents();
+  bool waited = false;
   const ScanSplit sp = scan_split(seq_lens, pl.B, N_max, upb, pl.scan_ctas);
-  if (c == 0 && tid == 0) {
-    for (int b = 0; b < pl.B; ++b)
-      if (seq_lens[b] < 0 || seq_lens[b] > N_max) atomicOr(status, kStatusSeqLen);
+  if (c >= sp.P_eff || sp.T == 0) {
+    pdl_wait();        // (the status word is cleared by the kernel before this one)
+    if (c == 0 && tid == 0)
+      for (int b = 0; b < pl.B; ++b)
+        if (seq_lens[b] < 0 || seq_lens[b] > N_max) atomicOr(status, kStatusSeqLen);
+    return;
   }
-  if (c >= sp.P_eff || sp.T == 0) return;
   long long lo = split_start(sp, c);
   const long long hi = split_start(sp, c + 1);
 
@@ -173,6 +185,18 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
   uint32_t lane_off[8];   // shared-window address of entry (z = 0, m = t ^ lx) for t = s & 7
 #pragma unroll
   for (int t = 0; t < 8; ++t) lane_off[t] = smem_u32(s_lut) + uint32_t((t ^ lx) * kEntryBytes);
+  // fp16 tables: 8-byte entries, a half warp per wavefront, so the skew runs over 16 subspaces:
+  // at step s the lane reads subspace (s & 16) + ((s & 15) ^ (lane & 15))
+  const uint32_t lxs = uint32_t(lane & 15) << 3;
+  const uint32_t hsel = 0x3210u ^ (uint32_t(lane & 3) * 0x1111u);      // byte order inside a word
+  const bool hswap1 = (lane & 4) != 0, hswap2 = (lane & 8) != 0;        // word order inside 16 bytes
+  // the fp16 table (64 KB: 256 rows of 256 bytes) starts at the first 64 KB boundary inside the
+  // 128 KB fp32 landing zone, so the lookup address is one xor of the table address, the row
+  // index shifted into place and the offsets below 256
+  const uint32_t lut_h = (smem_u32(s_lut) + 0xffffu) & ~0xffffu;
+  uint2* const s_lut_h = reinterpret_cast<uint2*>(smem_raw + (lut_h - smem_u32(s_lut)));
+  const uint32_t lane_h = lut_h ^ lxs;
+  static_assert(!kHalf || (M == 32 && GC == 4), "fp16 tables: M = 32, four heads per group");
 
   // locate the sequence that holds tile `lo`
   int b = 0;
@@ -204,15 +228,6 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     float* part = partials + (unit * pl.n_part + slot) * (size_t)(GC * (n_list + 2));
     float* part_sums = part + 2 * GC;
 
-    __syncthreads();   // previous segment's tables are no longer in use
-    if (tid == 0) {
-      const uint32_t lut_bytes_n = kLutFloats * 4;
-      const uint32_t co_bytes = pl.coarse_in_smem ? uint32_t(GC * n_list * 4) : 0u;
-      mbar_expect_tx(&s_bar, lut_bytes_n + co_bytes);
-      bulk_g2s(s_lut, lut + unit * (size_t)kLutFloats, lut_bytes_n, &s_bar);
-      if (co_bytes) bulk_g2s(s_coarse, g_coarse, co_bytes, &s_bar);
-      s_overflow = 0;
-    }
     for (int i = tid; i < GC * n_list; i += kScanThreads) part_sums[i] = 0.f;
 
     // prologue of the ring: the first kStages-1 tiles of this warp (overlaps the table copy)
@@ -223,9 +238,43 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
                       Nb, lane);
     TokenMeta cur;
     load_meta(cur, lids, norms, row_base, t * kTile + lane, t < tend && t * kTile + lane < Nb);
+    if (!waited) {                                  // the tables exist from here on
+      pdl_wait();
+      waited = true;
+      if (c == 0 && tid == 0)
+        for (int bb = 0; bb < pl.B; ++bb)
+          if (seq_lens[bb] < 0 || seq_lens[bb] > N_max) atomicOr(status, kStatusSeqLen);
+    }
+    __syncthreads();   // previous segment's tables are no longer in use
+    if (tid == 0) {
+      const uint32_t lut_bytes_n = kLutFloats * 4;
+      const uint32_t co_bytes = pl.coarse_in_smem ? uint32_t(GC * n_list * 4) : 0u;
+      mbar_expect_tx(&s_bar, lut_bytes_n + co_bytes);
+      bulk_g2s(s_lut, lut + unit * (size_t)kLutFloats, lut_bytes_n, &s_bar);
+      if (co_bytes) bulk_g2s(s_coarse, g_coarse, co_bytes, &s_bar);
+      s_overflow = 0;
+    }
     if (!mbar_wait(&s_bar, bar_parity)) atomicOr(status, kStatusCopyTimeout);
     bar_parity ^= 1u;
     __syncthreads();   // partial zeroed, tables landed
+    if constexpr (kHalf) {
+      // in place: every thread takes its 16 entries into registers, and only when all are read
+      // does anybody write the 8-byte versions over the first half of the same memory
+      constexpr int kPer = kCodes * M / kScanThreads;
+      float4 e[kPer];
+#pragma unroll
+      for (int u = 0; u < kPer; ++u) e[u] = reinterpret_cast<const float4*>(s_lut)[u * kScanThreads + tid];
+      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < kPer; ++u) {
+        const __half2 a = __floats2half2_rn(e[u].x, e[u].y), bq = __floats2half2_rn(e[u].z, e[u].w);
+        uint2 w;
+        w.x = *reinterpret_cast<const uint32_t*>(&a);
+        w.y = *reinterpret_cast<const uint32_t*>(&bq);
+        s_lut_h[u * kScanThreads + tid] = w;
+      }
+      __syncthreads();
+    }
 
     float mx[GC], ref2[GC];
 #pragma unroll
@@ -254,9 +303,48 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         Acc<GC> acc0, acc1;
         acc0.zero();
         acc1.zero();
-        // position p of the lane's code array <- original byte p ^ (lane & 7)
         uint32_t raw[M / 4], cw[M / 4];
         read_codes<M>(ring0 + (it % kStages) * CodeTile<M>::kBytes, lane, raw);
+        if constexpr (kHalf) {
+          // position p of every 16-byte group <- original byte p ^ (lane & 15)
+#pragma unroll
+          for (int q4 = 0; q4 < M / 16; ++q4) {
+            uint32_t r0 = raw[4 * q4], r1 = raw[4 * q4 + 1], r2 = raw[4 * q4 + 2], r3 = raw[4 * q4 + 3];
+            if (hswap1) { uint32_t t_ = r0; r0 = r1; r1 = t_; t_ = r2; r2 = r3; r3 = t_; }
+            if (hswap2) { uint32_t t_ = r0; r0 = r2; r2 = t_; t_ = r1; r1 = r3; r3 = t_; }
+            cw[4 * q4] = __byte_perm(r0, 0u, hsel); cw[4 * q4 + 1] = __byte_perm(r1, 0u, hsel);
+            cw[4 * q4 + 2] = __byte_perm(r2, 0u, hsel); cw[4 * q4 + 3] = __byte_perm(r3, 0u, hsel);
+          }
+          // four lookups are summed in fp16 (two levels), then widened and added in fp32
+#pragma unroll
+          for (int sb = 0; sb < M; sb += 4) {
+            unsigned long long v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int s = sb + u;
+              const uint32_t zrow = __byte_perm(cw[s >> 2], 0u, 0x4404u | (uint32_t(s & 3) << 4));   // z << 8
+              asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v[u])
+                           : "r"(zrow ^ lane_h ^ uint32_t(((s & 15) << 3) | ((s >> 4) << 7))));
+            }
+            uint32_t lo[4], hi[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { lo[u] = (uint32_t)v[u]; hi[u] = (uint32_t)(v[u] >> 32); }
+            uint32_t l01, l23, h01, h23, l4, h4;
+            asm("add.rn.f16x2 %0, %1, %2;" : "=r"(l01) : "r"(lo[0]), "r"(lo[1]));
+            asm("add.rn.f16x2 %0, %1, %2;" : "=r"(l23) : "r"(lo[2]), "r"(lo[3]));
+            asm("add.rn.f16x2 %0, %1, %2;" : "=r"(h01) : "r"(hi[0]), "r"(hi[1]));
+            asm("add.rn.f16x2 %0, %1, %2;" : "=r"(h23) : "r"(hi[2]), "r"(hi[3]));
+            asm("add.rn.f16x2 %0, %1, %2;" : "=r"(l4) : "r"(l01), "r"(l23));
+            asm("add.rn.f16x2 %0, %1, %2;" : "=r"(h4) : "r"(h01), "r"(h23));
+            const float2 fl = __half22float2(*reinterpret_cast<const __half2*>(&l4));
+            const float2 fh = __half22float2(*reinterpret_cast<const __half2*>(&h4));
+            Acc<GC> w;
+            w.lo = (unsigned long long)__float_as_uint(fl.x) | ((unsigned long long)__float_as_uint(fl.y) << 32);
+            w.hi = (unsigned long long)__float_as_uint(fh.x) | ((unsigned long long)__float_as_uint(fh.y) << 32);
+            if (sb & 4) acc1.merge(w); else acc0.merge(w);
+          }
+        } else {
+        // position p of the lane's code array <- original byte p ^ (lane & 7)
 #pragma unroll
         for (int j = 0; j < M / 8; ++j) {
           const uint32_t a = raw[2 * j], bb = raw[2 * j + 1];
@@ -277,6 +365,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
             acc0.merge(v[u]);
             acc1.merge(v[u + 1]);
           }
+        }
         }
         acc0.merge(acc1);
         float accf[GC], co[GC];
@@ -409,15 +498,15 @@ size_t scan_smem_bytes(const Plan& pl, bool coarse_in_smem, int stages) {
   return tables + (size_t)(kScanThreads / 32) * stages * kTile * pl.code_bytes;
 }
 
-template <int M, int GC, int S>
+template <int M, int GC, int S, bool kHalf = false>
 static cudaError_t launch_scan_t(const Plan& pl, const pqhsa_index& ix, const float* lut,
                                  const float* coarse, const int32_t* seq_lens, float* scores,
                                  float* partials, int* status, cudaStream_t st) {
   const size_t smem = scan_smem_bytes(pl, pl.coarse_in_smem != 0, S);
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S>,
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<M, GC, S, kHalf>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_pdl(scan_kernel<M, GC, S>, dim3(pl.scan_ctas), dim3(kScanThreads), smem, st, pl,
+  return launch_pdl(scan_kernel<M, GC, S, kHalf>, dim3(pl.scan_ctas), dim3(kScanThreads), smem, st, pl,
                     ix.codes, ix.list_ids, ix.key_norms, lut, coarse, seq_lens, scores, partials,
                     status);
 }
@@ -427,6 +516,12 @@ cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,
                         float* list_partials, int* status, cudaStream_t st) {
   if (pl.n_code == 16)
     return launch_scan4(pl, ix, lut, coarse, seq_lens, scores, list_partials, status, st);
+  if (pl.half_tables) {
+    if (pl.M != 32 || pl.Gc != 4) return cudaErrorInvalidValue;          // (rejected by make_plan)
+    if (pl.scan_stages >= 3)
+      return launch_scan_t<32, 4, 3, true>(pl, ix, lut, coarse, seq_lens, scores, list_partials, status, st);
+    return launch_scan_t<32, 4, 2, true>(pl, ix, lut, coarse, seq_lens, scores, list_partials, status, st);
+  }
 #define PQHSA_SCAN_CASE(MM, GG)                                                               \
   if (pl.M == MM && pl.Gc == GG) {                                                            \
     if (pl.scan_stages >= 3)                                                                  \

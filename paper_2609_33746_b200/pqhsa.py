@@ -47,7 +47,8 @@ class Params(ctypes.Structure):
         "max_seq_len", "page_size", "max_pages_per_seq", "n_sink", "n_local")] + [
         ("budget_ppm", ctypes.c_uint32), ("k_max", ctypes.c_int32), ("sm_scale", ctypes.c_float),
         ("dtype", ctypes.c_int32), ("exact_set_multiple", ctypes.c_int32),
-        ("variant", ctypes.c_int32), ("indexed_lens", ctypes.c_void_p)]
+        ("variant", ctypes.c_int32), ("table_precision", ctypes.c_int32),
+        ("indexed_lens", ctypes.c_void_p)]
 
 
 class Index(ctypes.Structure):
@@ -143,7 +144,7 @@ def _stream(stream) -> Optional[int]:
 def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_pages_per_seq,
                 budget_ppm, dtype, head_dim=128, pq_ncode=256, page_size=16, n_sink=0, n_local=0,
                 k_max=None, sm_scale=None, exact_set_multiple=0, variant="B",
-                indexed_lens=None) -> Params:
+                indexed_lens=None, fp16_tables=False) -> Params:
     """`indexed_lens`: device int32 tensor [batch] or None; the caller keeps it alive."""
     if k_max is None:
         k_max = max(1, (max_seq_len * budget_ppm + 999_999) // 1_000_000)
@@ -154,7 +155,8 @@ def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_
     code = {"fp16": F16, "bf16": BF16, torch.float16: F16, torch.bfloat16: BF16}[dtype]
     return Params(batch, n_q_heads, n_kv_heads, head_dim, n_list, pq_m, head_dim // pq_m, pq_ncode,
                   max_seq_len, page_size, max_pages_per_seq, n_sink, n_local, budget_ppm, k_max,
-                  sm_scale, code, exact_set_multiple, VARIANTS[variant], _ptr(indexed_lens))
+                  sm_scale, code, exact_set_multiple, VARIANTS[variant], 1 if fp16_tables else 0,
+                  _ptr(indexed_lens))
 
 
 def make_index(centroids, codebooks, codes, list_ids, key_norms, list_vmeans,

@@ -13,7 +13,8 @@ class DecodeOp:
     """Device buffers + marshalled structs of one workload; every method is one library call."""
 
     def __init__(self, inp: DecodeInputs, index: IvfPqIndex, device: str = "cuda:0",
-                 budget_ppm: int | None = None, variant: str | None = None):
+                 budget_ppm: int | None = None, variant: str | None = None,
+                 fp16_tables: bool = False):
         cfg: DecodeConfig = inp.cfg
         self.cfg, self.device = cfg, torch.device(device)
         dev = self.device
@@ -47,7 +48,8 @@ class DecodeOp:
             max_pages_per_seq=inp.max_pages_per_seq, budget_ppm=ppm, dtype=cfg.dtype,
             head_dim=cfg.head_dim, pq_ncode=cfg.pq_ncode, page_size=cfg.page_size, n_sink=cfg.n_sink,
             n_local=cfg.n_local, exact_set_multiple=cfg.exact_set_multiple,
-            variant=cfg.variant if variant is None else variant, indexed_lens=self.indexed_lens)
+            variant=cfg.variant if variant is None else variant, indexed_lens=self.indexed_lens,
+            fp16_tables=fp16_tables)
         self.index = pqhsa.make_index(self.centroids, self.codebooks, self.codes, self.list_ids,
                                       self.key_norms, self.list_vmeans, self.list_counts)
         self.kv = pqhsa.make_paged_kv(self.k_cache, self.v_cache, inp.stride_page,

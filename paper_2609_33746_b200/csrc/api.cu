@@ -115,7 +115,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.hist_chunks = 2 * o.rows <= sel_slots ? sel_slots / o.rows : ceil_div(2LL * sel_slots, o.rows);
   if (o.hist_chunks > ceil_div(o.N_max, kSelChunk)) o.hist_chunks = ceil_div(o.N_max, kSelChunk);
   if (o.hist_chunks < 1) o.hist_chunks = 1;
-  o.cand_cap = o.N_max / 4 > kSelChunk ? o.N_max / 4 : kSelChunk;
+  o.cand_cap = o.N_max / 8 > kSelChunk ? o.N_max / 8 : kSelChunk;
   if (o.cand_cap > o.N_max) o.cand_cap = o.N_max;
   // attend kernel, background CTAs per (sequence, KV head, head group): about two per SM in
   // total, at least 32 lists each
@@ -182,7 +182,7 @@ void make_layout(const Plan& pl, WsLayout* L) {
   L->attend_zero_bytes = o - L->attend_tickets;
   L->zero_bytes = o - L->zero_begin;
   L->rowstate = take((size_t)pl.rows * 16);
-  L->cand = take((size_t)pl.rows * pl.cand_cap * 4);
+  L->cand = take((size_t)pl.rows * pl.cand_cap * 8);
   L->bg_max = take((size_t)pl.rows * 4);
   L->split_part = take((size_t)pl.rows * attend_parts(pl) * (4 + kHeadDim) * 4);
   L->stage_end = o;

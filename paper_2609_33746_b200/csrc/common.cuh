@@ -64,7 +64,7 @@ struct WsLayout {
   size_t attend_tickets;             // uint32 [rows]
   size_t attend_zero_bytes;          // tickets + bg_mass: what the attend stage needs cleared
   size_t rowstate;                   // int32  [rows][4]: lo, hi (float bits), k, n
-  size_t cand;                       // int32  [rows][cand_cap]: candidate positions
+  size_t cand;                       // uint2  [rows][cand_cap]: candidates as (score key, position)
   size_t bg_mass;                    // float  [rows][n_list]: M_j relative to bg_max (accumulated)
   size_t bg_aux;                     // float  [rows][4]: [0] sum of the selected tokens' approximate logits
   size_t bg_tcount;                  // int32  [rows][n_list]: selected tokens per list (variant Bx only)

@@ -2,19 +2,20 @@
 // T(q) = TopK_{k, i in R} l~_i with k = ceil(rho |R|).
 //
 // One pass over the scores instead of a multi-pass radix sort of the whole row:
-//   sample kernel  one CTA per row reads 4096 scores (1024 groups of 4, jittered stride)
-//                  and takes two order statistics of the sample that bracket the k-th largest
-//                  score of the row with a 6-sigma margin: lo <= s_k <= hi (one histogram of
-//                  the sample over 4096 equal buckets of its range; the bracket's edges are
-//                  bucket edges);
+//   sample kernel  one CTA per row reads up to 16384 scores (1024 groups of 16 at a jittered
+//                  stride; never more than a quarter of the row) and takes two order
+//                  statistics of the sample that bracket the k-th largest score of the row
+//                  with a 6-sigma margin: lo <= s_k <= hi (one histogram of the sample over
+//                  4096 equal buckets of its range; the bracket's edges are bucket edges).  At
+//                  a 1 % budget and 128K tokens about half of the k winners lie above hi;
 //   filter kernel  scores above hi are certain winners and are written out at once; scores in
-//                  [lo, hi] (a few percent of k) are appended to a candidate list; the last
-//                  CTA of the row (atomic ticket, nobody waits) checks the bracket by counting
-//                  (#winners <= k <= #winners + #candidates) and finishes exactly: one
-//                  histogram of the candidates over 4096 equal buckets of [lo, hi], everything
-//                  above the bucket of the k-th largest is taken, the few items inside it are
-//                  ranked against each other (a 12/12/8-bit radix select remains for candidate
-//                  sets that do not fit shared memory or pile up in one bucket).
+//                  [lo, hi] are appended, as (key, position) pairs, to a candidate list; the
+//                  last CTA of the row (atomic ticket, nobody waits) checks the bracket by
+//                  counting (#winners <= k <= #winners + #candidates) and finishes exactly:
+//                  one histogram of the candidates over 4096 equal buckets of their range,
+//                  everything above the bucket of the k-th largest is taken, the few items
+//                  inside it are ranked against each other (a 12/12/8-bit radix select remains
+//                  for candidate sets that do not fit shared memory or pile up in one bucket).
 // If the bracket misses (a row whose order defeats the sample), that last CTA redoes the
 // row from the scores themselves with the same radix select, so the result is always the
 // exact top-k; equal scores at the threshold are taken in order of position (lowest first),
@@ -28,9 +29,9 @@ namespace {
 constexpr int kElems = kSelChunk / kSelThreads;   // scores per thread per chunk (16)
 constexpr int kStashCap = 5120;                   // candidates resolved from shared memory
 constexpr int kFilterSmemBytes = kHistBins * 4 + kStashCap * 8;   // dynamic: above the 48 KB static limit
-constexpr int kSample = 4096;                     // sampled scores per row
-constexpr int kSamplePer = kSample / kSelThreads; // per thread (8)
-constexpr int kSampleGroups = kSample / 4;        // groups of 4 consecutive scores
+constexpr int kSample = 16384;                    // sampled scores per row (at most a quarter of it)
+constexpr int kSamplePer = kSample / kSelThreads; // per thread (32)
+constexpr int kSampleGroups = kSample / 16;       // groups of 16 consecutive scores (64 bytes)
 constexpr float kBracketSigmas = 6.0f;
 
 // rowstate: [0] lo, [1] hi (float bits), [2] k, [3] n
@@ -219,18 +220,23 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
   } else if (k == rg.r_end - rg.r_begin) {
     hi = -CUDART_INF_F;                            // all of R: every score above -inf is a winner
   } else if (n > kSelChunk) {
-    // 1024 aligned groups of 4 consecutive scores; group g sits in the g-th of 1024 equal
-    // strides of the row at a hashed offset (reads 16 bytes per touched 32-byte sector)
+    // n_groups aligned groups of 16 consecutive scores (1024 of them on a long row, never more
+    // than a quarter of the row); group g sits in the g-th of n_groups equal strides of the
+    // row at a hashed offset, and four neighbouring threads read its 64 bytes
     const float* rs = scores + (size_t)row * pl.N_max;
+    const int n_groups = min(kSampleGroups, n / 64);
     float s[kSamplePer];
 #pragma unroll
     for (int u = 0; u < kSamplePer / 4; ++u) {
-      const int g = u * kSelThreads + tid;
-      const long long a = (long long)g * n / kSampleGroups, z = (long long)(g + 1) * n / kSampleGroups;
-      const uint32_t h = (uint32_t)g * 2654435761u;
-      long long off = (a + (long long)((h >> 8) % (uint32_t)(z - a))) & ~3LL;
-      if (off + 4 > n) off = (n - 4) & ~3LL;
-      const float4 f = __ldcg(reinterpret_cast<const float4*>(rs + off));
+      const int g = (u * kSelThreads + tid) >> 2, part = tid & 3;
+      float4 f = make_float4(CUDART_NAN_F, CUDART_NAN_F, CUDART_NAN_F, CUDART_NAN_F);   // not sampled
+      if (g < n_groups) {
+        const long long a = (long long)g * n / n_groups, z = (long long)(g + 1) * n / n_groups;
+        const uint32_t h = (uint32_t)g * 2654435761u;
+        long long off = (a + (long long)((h >> 8) % (uint32_t)(z - a))) & ~15LL;
+        if (off + 16 > n) off = (n - 16) & ~15LL;
+        f = __ldcg(reinterpret_cast<const float4*>(rs + off) + part);
+      }
       s[4 * u] = f.x; s[4 * u + 1] = f.y; s[4 * u + 2] = f.z; s[4 * u + 3] = f.w;
     }
     for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;   // while the loads fly
@@ -251,11 +257,12 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
     __syncthreads();
 #pragma unroll
     for (int w = 0; w < kSelThreads / 32; ++w) { mn = fminf(mn, s_mm[0][w]); mx = fmaxf(mx, s_mm[1][w]); }
-    // the k-th largest of the row sits near rank p*4096 of the sample; the bracket is
+    // the k-th largest of the row sits near rank p * n_sample of the sample; the bracket is
     // +- 6 sigma of that count (binomial bound on the hypergeometric spread), + 2
+    const int n_sample = 16 * n_groups;
     const float p = (float)k / (float)n;
-    const float r = p * kSample;
-    const int mgn = (int)ceilf(kBracketSigmas * sqrtf(kSample * p * (1.f - p))) + 2;
+    const float r = p * n_sample;
+    const int mgn = (int)ceilf(kBracketSigmas * sqrtf(n_sample * p * (1.f - p))) + 2;
     const int r_hi = (int)floorf(r) - mgn, r_lo = (int)ceilf(r) + mgn;
     if (mx > mn) {
       // one histogram of the samples over 4096 equal buckets of [mn, mx] (non-finite samples
@@ -264,13 +271,14 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
       // Whatever the bracket is, the filter kernel checks it by counting.
       const float scale = (float)kHistBins / (mx - mn);
 #pragma unroll
-      for (int e = 0; e < kSamplePer; ++e) atomicAdd(&s_hist[linear_bucket(s[e], mn, scale)], 1u);
+      for (int e = 0; e < kSamplePer; ++e)
+        if (s[e] == s[e]) atomicAdd(&s_hist[linear_bucket(s[e], mn, scale)], 1u);
       __syncthreads();
       int b_hi, b_lo;
-      find_two_buckets(s_hist, max(r_hi, 0), min(r_lo, kSample - 1), s_scan, b_hi, b_lo);
+      find_two_buckets(s_hist, max(r_hi, 0), min(r_lo, n_sample - 1), s_scan, b_hi, b_lo);
       const float width = (mx - mn) / (float)kHistBins;
       if (r_hi >= 0) hi = mn + (float)(b_hi + 2) * width;
-      if (r_lo < kSample && b_lo >= 2) lo = mn + (float)(b_lo - 1) * width;
+      if (r_lo < n_sample && b_lo >= 2) lo = mn + (float)(b_lo - 1) * width;
     } else if (mx == mn) {
       hi = mx;                                     // all finite samples equal: take that value
       lo = mn;                                     // as the whole bracket
@@ -290,11 +298,11 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
 enum Source { kFromStash = 0, kFromList = 1, kFromRow = 2 };
 
 // Calls f(valid, key, position) for every item of the source: the candidates staged in
-// shared memory as (key, position), the candidate list in global memory (positions; the key
-// comes from the score row), or the whole score row.  Uniform trip
+// shared memory as (key, position), the candidate list in global memory (the same pairs),
+// or the whole score row.  Uniform trip
 // count: f may use warp votes.
 template <class F>
-__device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, const int32_t* cand,
+__device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, const uint2* cand,
                                               int n_items, const float* rs, F f) {
   const int tid = threadIdx.x;
   constexpr int U = 4;
@@ -307,19 +315,16 @@ __device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, con
     }
   } else if (src == kFromList) {
     for (int base = 0; base < n_items; base += kSelThreads * U) {
-      int pos[U];
-      float sc[U];
+      uint2 it[U];
       bool v[U];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int i = base + u * kSelThreads + tid;
         v[u] = i < n_items;
-        pos[u] = v[u] ? __ldcg(cand + i) : 0;
+        it[u] = v[u] ? __ldcg(cand + i) : make_uint2(0u, 0u);
       }
 #pragma unroll
-      for (int u = 0; u < U; ++u) sc[u] = v[u] ? __ldcg(rs + pos[u]) : 0.f;
-#pragma unroll
-      for (int u = 0; u < U; ++u) f(v[u], score_key(sc[u]), pos[u]);
+      for (int u = 0; u < U; ++u) f(v[u], it[u].x, (int)it[u].y);
     }
   } else {
     for (int base = 0; base < n_items; base += kSelThreads * U) {
@@ -340,7 +345,7 @@ __device__ __forceinline__ void for_each_item(int src, const uint2* s_stash, con
 // Exact selection of the `r` largest of the source's items (ties: lowest position), appended
 // to out[base_out ...].  Radix digits 12 / 12 / 8.  Returns the key of the r-th largest.
 // Runs in one CTA; 1 <= r <= n_items.
-__device__ uint32_t resolve_top_r(int src, const uint2* s_stash, const int32_t* cand, int n_items,
+__device__ uint32_t resolve_top_r(int src, const uint2* s_stash, const uint2* cand, int n_items,
                                   const float* rs, int n, int r, int32_t* out, uint32_t base_out,
                                   int k_max, uint32_t* s_hist, int* s_scan, uint32_t* s_emit) {
   const int tid = threadIdx.x;
@@ -408,7 +413,7 @@ __device__ uint32_t resolve_top_r(int src, const uint2* s_stash, const int32_t* 
 
 __global__ void __launch_bounds__(kSelThreads, 3)
 sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restrict__ counters,
-                  const int32_t* __restrict__ rowstate, int32_t* __restrict__ cand,
+                  const int32_t* __restrict__ rowstate, uint2* __restrict__ cand,
                   int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_count,
                   float* __restrict__ kth, int* __restrict__ status) {
   // main pass: a 512-entry hit buffer per warp; last CTA: histogram + candidate stash.
@@ -430,7 +435,7 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
   if (k == 0) return;
   const float* rs = scores + (size_t)row * pl.N_max;
   int32_t* out = sel_idx + (size_t)row * pl.k_max;
-  int32_t* rc = cand + (size_t)row * pl.cand_cap;
+  uint2* rc = cand + (size_t)row * pl.cand_cap;          // (key, position) pairs
   uint32_t* n_out = &counters[row * 4 + 2];
   uint32_t* n_cand = &counters[row * 4 + 3];
 
@@ -473,8 +478,10 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
         if (p < (uint32_t)pl.k_max) out[p] = (int)(ent & 0x7fffffffu);
       }
       if (is_cnd) {
+        // the score comes back from L2 (this warp read it a moment ago), so that the row's
+        // last CTA finds key and position together and has no dependent gather to wait for
         const uint32_t p = bc + __popc(mc & lt);
-        if (p < (uint32_t)pl.cand_cap) rc[p] = (int)ent;
+        if (p < (uint32_t)pl.cand_cap) rc[p] = make_uint2(score_key(__ldcg(rs + ent)), ent);
       }
       bw += __popc(mw);
       bc += __popc(mc);
@@ -546,35 +553,55 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
       __syncthreads();
     } else {
       int src = kFromList;
+      uint32_t kmin = 0xffffffffu, kmax = 0u;                  // range of the finite staged keys
       if (C <= kStashCap) {
         constexpr int kPer = kStashCap / kSelThreads;          // 10: all loads issued together
-        int pos[kPer];
-        float sc[kPer];
+        uint2 it[kPer];
 #pragma unroll
         for (int u = 0; u < kPer; ++u) {
           const int i = u * kSelThreads + tid;
-          pos[u] = i < C ? __ldcg(rc + i) : -1;
+          it[u] = i < C ? __ldcg(rc + i) : make_uint2(0x80000000u, 0u);
         }
 #pragma unroll
-        for (int u = 0; u < kPer; ++u) sc[u] = pos[u] >= 0 ? __ldcg(rs + pos[u]) : 0.f;
+        for (int u = 0; u < kPer; ++u) {
+          const int i = u * kSelThreads + tid;
+          if (i < C) {
+            s_stash[i] = it[u];
+            if (fabsf(key_score(it[u].x)) < CUDART_INF_F) {
+              kmin = min(kmin, it[u].x);
+              kmax = max(kmax, it[u].x);
+            }
+          }
+        }
 #pragma unroll
-        for (int u = 0; u < kPer; ++u)
-          if (pos[u] >= 0)
-            s_stash[u * kSelThreads + tid] = make_uint2(score_key(sc[u]), (uint32_t)pos[u]);
+        for (int o = 16; o > 0; o >>= 1) {
+          kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+          kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+        }
+        if (lane == 0) { s_scan[warp] = (int)kmin; s_scan[16 + warp] = (int)kmax; }
         __syncthreads();
+#pragma unroll
+        for (int w = 0; w < kSelThreads / 32; ++w) {
+          kmin = min(kmin, (uint32_t)s_scan[w]);
+          kmax = max(kmax, (uint32_t)s_scan[16 + w]);
+        }
+        __syncthreads();                                       // s_scan is reused below
         src = kFromStash;
       }
       bool done = false;
-      if (src == kFromStash && lo_f > -CUDART_INF_F && hi_f < CUDART_INF_F && hi_f > lo_f) {
-        // Fast finish.  The staged candidates all lie in [lo, hi]: ONE histogram over 4096
-        // equal buckets of that interval finds the bucket of the r-th largest; everything in a
-        // higher bucket is taken at once, and the few items of that bucket are ranked against
-        // each other (larger score first, then lower position: the stable rule).
-        const float scale = (float)kHistBins / (hi_f - lo_f);
+      if (src == kFromStash && kmax > kmin) {
+        // Fast finish.  ONE histogram of the staged candidates over 4096 equal buckets of the
+        // range of their finite scores (candidates at -inf, the sink and window positions of a
+        // row that was not bracketed from below, fall into the bottom bucket) finds the bucket of
+        // the r-th largest; everything in a higher bucket is taken at once, and the few items of
+        // that bucket are ranked against each other (larger score first, then lower position:
+        // the stable rule).
+        const float lo_h = key_score(kmin);
+        const float scale = (float)kHistBins / (key_score(kmax) - lo_h);
         for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
         __syncthreads();
         for (int i = tid; i < C; i += kSelThreads)
-          atomicAdd(&s_hist[linear_bucket(key_score(s_stash[i].x), lo_f, scale)], 1u);
+          atomicAdd(&s_hist[linear_bucket(key_score(s_stash[i].x), lo_h, scale)], 1u);
         __syncthreads();
         int d, above;
         find_digit(s_hist, kHistBins, r, s_scan, d, above);
@@ -589,7 +616,7 @@ sel_filter_kernel(Plan pl, const float* __restrict__ scores, uint32_t* __restric
             const int i = base + tid;
             const bool v = i < C;
             const uint2 it = v ? s_stash[i] : make_uint2(0u, 0u);
-            const int bk = v ? linear_bucket(key_score(it.x), lo_f, scale) : -1;
+            const int bk = v ? linear_bucket(key_score(it.x), lo_h, scale) : -1;
             const int p = warp_append(v && bk > d, &s_emit);
             if (p >= 0 && (uint32_t)W + p < (uint32_t)pl.k_max) out[W + p] = (int)it.y;
             if (v && bk == d) tie[atomicAdd(&s_tie, 1u)] = it;
@@ -638,7 +665,7 @@ cudaError_t launch_select(const Plan& pl, const WsLayout& L, char* ws, const flo
                           float* kth, cudaStream_t st) {
   uint32_t* counters = reinterpret_cast<uint32_t*>(ws + L.counters);
   int32_t* rowstate = reinterpret_cast<int32_t*>(ws + L.rowstate);
-  int32_t* cand = reinterpret_cast<int32_t*>(ws + L.cand);
+  uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
   int* status = reinterpret_cast<int*>(ws + L.status);
   cudaError_t e = launch_pdl(sel_sample_kernel, dim3(pl.rows), dim3(kSelThreads), 0, st, pl, scores,
                              seq_lens, rowstate, sel_count, kth);

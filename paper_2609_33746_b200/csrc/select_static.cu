@@ -55,7 +55,7 @@ void make_select_layout(const Plan& pl, WsLayout* L) {
   L->counters = take((size_t)pl.rows * 16);
   L->zero_bytes = o;
   L->rowstate = take((size_t)pl.rows * 16);
-  L->cand = take((size_t)pl.rows * pl.cand_cap * 4);
+  L->cand = take((size_t)pl.rows * pl.cand_cap * 8);
   L->stage_end = o;
   L->total = o;
 }

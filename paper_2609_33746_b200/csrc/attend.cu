@@ -60,7 +60,7 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
     return;
   }
   // the selected tokens of this CTA's slice: start their gathers first
-  const int cnt = sel_count[row];
+  const int cnt = min(max(sel_count[row], 0), pl.k_max);   // (a count outside [0, k_max] is not followed)
   const int tl = (int)((long long)c * cnt / C), th = (int)((long long)(c + 1) * cnt / C);
   const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
   const float* rs = scores + (size_t)row * pl.N_max;
@@ -305,7 +305,7 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
           const int row = row0 + g;
           const int n_seq = clamp_len(seq_lens[b], pl.N_max);
           const Region rg = region_of(pl, n_seq, b);
-          const int k_sel = sel_count[row];
+          const int k_sel = min(max(sel_count[row], 0), pl.k_max);
           Z_c = (float)max(0, rg.r_end - rg.r_begin - k_sel);
           if (k_sel <= 0 || !(bg_max[row] > -CUDART_INF_F)) Z_c = 0.f;   // no T: no shared logit
           if (variant == PQHSA_VARIANT_C2) m_c = (k_sel > 0 ? bg_aux[row * 4] / (float)k_sel : 0.f) * kLog2e;
@@ -343,7 +343,7 @@ attend_kernel(Plan pl, const T* __restrict__ q, const T* __restrict__ kc, const 
   pdl_launch_dependents();
   // the exact set E = T u S u L (Sec. 3.2), as one index space: the selected tokens first,
   // then the sink prefix, then the local window
-  const int cnt = sel_count[row];
+  const int cnt = min(max(sel_count[row], 0), pl.k_max);   // (a count outside [0, k_max] is not followed)
   const int n_seq = clamp_len(seq_lens[b], pl.N_max);
   const Region rg = region_of(pl, n_seq, b);
   const int n_s = rg.r_begin, n_exact = cnt + n_s + (n_seq - rg.r_end);
@@ -521,7 +521,7 @@ bx_corr_kernel(Plan pl, const T* __restrict__ vc, long long stride_page, long lo
   pdl_wait();               // (nothing above this line may return: see the file header)
   pdl_launch_dependents();
   const int n_seq = clamp_len(seq_lens[b], pl.N_max);
-  const int cnt = sel_count[row];
+  const int cnt = min(max(sel_count[row], 0), pl.k_max);   // (a count outside [0, k_max] is not followed)
   const int tl = (int)((long long)split * cnt / S), th = (int)((long long)(split + 1) * cnt / S);
   const int32_t* sel = sel_idx + (size_t)row * pl.k_max;
   const size_t ukv = (size_t)b * pl.Hkv + kv;

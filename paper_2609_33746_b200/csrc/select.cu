@@ -209,37 +209,40 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
   __shared__ float s_mm[2][kSelThreads / 32];
   const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = row / pl.Hq;
-  pdl_wait();
-  pdl_launch_dependents();
+  // what depends on the call's inputs only (row length, budget, sample offsets, the cleared
+  // histogram) is done before the wait for the scan's scores
   const int n = clamp_len(seq_lens[b], pl.N_max);
   const int k = region_budget(pl, n, b);
   const Region rg = region_of(pl, n, b);
+  // n_groups aligned groups of 16 consecutive scores (1024 of them on a long row, never more
+  // than a quarter of the row); group g sits in the g-th of n_groups equal strides of the
+  // row at a hashed offset, and four neighbouring threads read its 64 bytes
+  const int n_groups = min(kSampleGroups, n / 64);
+  const uint32_t stride = n_groups > 0 ? (uint32_t)n / (uint32_t)n_groups : 0u;     // >= 64
+  int off[kSamplePer / 4];
+#pragma unroll
+  for (int u = 0; u < kSamplePer / 4; ++u) {
+    const int g = (u * kSelThreads + tid) >> 2;
+    const uint32_t h = (uint32_t)g * 2654435761u;
+    off[u] = g < n_groups ? (int)min(((uint32_t)g * stride + __umulhi(h, stride)) & ~15u, (uint32_t)(n - 16) & ~15u) + 4 * (tid & 3) : -1;
+  }
+  for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
+  pdl_wait();
+  pdl_launch_dependents();
   float lo = -CUDART_INF_F, hi = CUDART_INF_F;     // default: every score is a candidate
   if (k == 0) {
     if (tid == 0) { sel_count[row] = 0; kth[row] = CUDART_NAN_F; }
   } else if (k == rg.r_end - rg.r_begin) {
     hi = -CUDART_INF_F;                            // all of R: every score above -inf is a winner
   } else if (n > kSelChunk) {
-    // n_groups aligned groups of 16 consecutive scores (1024 of them on a long row, never more
-    // than a quarter of the row); group g sits in the g-th of n_groups equal strides of the
-    // row at a hashed offset, and four neighbouring threads read its 64 bytes
     const float* rs = scores + (size_t)row * pl.N_max;
-    const int n_groups = min(kSampleGroups, n / 64);
     float s[kSamplePer];
 #pragma unroll
     for (int u = 0; u < kSamplePer / 4; ++u) {
-      const int g = (u * kSelThreads + tid) >> 2, part = tid & 3;
       float4 f = make_float4(CUDART_NAN_F, CUDART_NAN_F, CUDART_NAN_F, CUDART_NAN_F);   // not sampled
-      if (g < n_groups) {
-        const long long a = (long long)g * n / n_groups, z = (long long)(g + 1) * n / n_groups;
-        const uint32_t h = (uint32_t)g * 2654435761u;
-        long long off = (a + (long long)((h >> 8) % (uint32_t)(z - a))) & ~15LL;
-        if (off + 16 > n) off = (n - 16) & ~15LL;
-        f = __ldcg(reinterpret_cast<const float4*>(rs + off) + part);
-      }
+      if (off[u] >= 0) f = __ldcg(reinterpret_cast<const float4*>(rs + off[u]));
       s[4 * u] = f.x; s[4 * u + 1] = f.y; s[4 * u + 2] = f.z; s[4 * u + 3] = f.w;
     }
-    for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;   // while the loads fly
     // range of the finite samples (sink and window positions hold -inf)
     float mn = CUDART_INF_F, mx = -CUDART_INF_F;
 #pragma unroll

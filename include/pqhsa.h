@@ -81,7 +81,8 @@ typedef struct {
   int32_t variant;            /* pqhsa_variant: how the background term is formed (Table 2);  */
                               /* 0 = PQ-HSA itself                                            */
   int32_t table_precision;    /* pqhsa_table_precision: 0 = fp32 lookup tables (the mode every  */
-                              /* stated tolerance refers to), 1 = fp16 tables in the scan        */
+                              /* stated tolerance refers to), 1 = fp16 tables in the scan, 2 =   */
+                              /* fp16 tables and an fp32 re-score of the top-k's threshold zone  */
   const int32_t* indexed_lens;/* DEVICE pointer [B] or NULL.  Number of leading positions of  */
                               /* each sequence that the index covers: R_b = [|S_b|,           */
                               /* indexed_lens[b]) and L_b = everything after (Sec. 3.3: a new */
@@ -97,8 +98,15 @@ typedef struct {
  * entries' magnitude instead of fp32 rounding.  Everything downstream is unchanged: the top-k is
  * exact on those scores, the selected tokens are attended with exact logits, and the list sums use
  * the same approximate logits that are later taken out of them.  v1: pq_ncode == 256, pq_m == 32,
- * G >= 3 (groups of four heads). */
-typedef enum { PQHSA_TABLES_FP32 = 0, PQHSA_TABLES_FP16 = 1 } pqhsa_table_precision;
+ * G >= 3 (groups of four heads).
+ * PQHSA_TABLES_FP16_RESCORE adds the usual second stage of such scans: the tokens whose approximate
+ * score lies within the table-rounding bound of the k-th one are scored again from the fp32 tables and
+ * the top-k is re-decided among them (pqhsa_rescore), so that the selected set is the one the fp32
+ * tables give (equal fp32 scores: lower position first) and kth_score is the exact k-th fp32 score.
+ * The score rows and the list sums keep the fp16-table values. */
+typedef enum {
+  PQHSA_TABLES_FP32 = 0, PQHSA_TABLES_FP16 = 1, PQHSA_TABLES_FP16_RESCORE = 2
+} pqhsa_table_precision;
 
 /* Mechanism variants of the paper's ablation (Table 2; App. B, "Variant definitions").  All of
  * them keep the selector, the budget and the exact part; they differ in the background term.
@@ -209,6 +217,18 @@ int pqhsa_scan(const pqhsa_params* params, const pqhsa_index* index, const float
 int pqhsa_select(const pqhsa_params* params, const float* scores, const int32_t* seq_lens,
                  int32_t* sel_idx, int32_t* sel_count, float* kth_score,
                  void* ws, size_t ws_bytes, void* stream);
+
+/* Step 3b, table_precision == PQHSA_TABLES_FP16_RESCORE only (PQHSA_ERR_INVALID_ARG otherwise): the
+ * fp32 re-score of the threshold zone.  Call after pqhsa_select with the SAME `ws` that pqhsa_scan and
+ * pqhsa_select were given (it holds the segment norms of the scan and the candidate lists of the
+ * top-k) and with their lut / coarse / scores / sel_idx / sel_count / kth_score.  Replaces in sel_idx
+ * the positions that the fp32 tables rank out of the top-k by those they rank in, and sets kth_score
+ * to the k-th largest fp32-table score.  A row whose threshold zone holds more than 1024 tokens keeps
+ * its approximate top-k and sets bit 64 of the device status word.  One launch on `stream`. */
+int pqhsa_rescore(const pqhsa_params* params, const pqhsa_index* index, const float* lut,
+                  const float* coarse, const float* scores, const int32_t* seq_lens,
+                  int32_t* sel_idx, const int32_t* sel_count, float* kth_score, void* ws,
+                  size_t ws_bytes, void* stream);
 
 /* Step 4 (Eq. 4-5).  Gathers the K/V rows of the exact set E_b = S_b u L_b u T (sinks, window,
  * selected tokens) from the paged cache and attends them with exact logits, takes the
@@ -330,7 +350,8 @@ int pqhsa_decode_host(const pqhsa_params* params, const void* q_host, void* q_de
 /* Reads the status word kernels set when they meet an inconsistency: copies it to the host and
  * waits for `stream`.  Returns PQHSA_OK or PQHSA_ERR_DEVICE_CHECK.  Valid after pqhsa_scan /
  * pqhsa_select / pqhsa_hybrid_attend / pqhsa_decode on the same ws.  Bits: 1 selected count != k,
- * 2 seq_len outside [0, max_seq_len], 4 a bounded wait on a bulk copy ran out; a library built
+ * 2 seq_len outside [0, max_seq_len], 4 a bounded wait on a bulk copy ran out, 64 a row kept its
+ * approximate top-k in the re-score pass (see pqhsa_rescore); a library built
  * with -DPQHSA_DEBUG (pqhsa_debug_build() == 1) also records the indices that the release
  * build silently clamps or skips: 8 list id >= n_list, 16 selected position outside the indexed
  * region, 32 negative page id.  No check traps: the CUDA context stays usable. */

@@ -12,7 +12,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libpqhsa.so")
 SOURCES = ["api.cu", "lut.cu", "scan.cu", "scan4.cu", "select.cu", "attend.cu", "select_static.cu", "dense.cu",
-           "update.cu", "build.cu"]
+           "update.cu", "build.cu", "rescore.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
               "-I", CSRC]

@@ -50,7 +50,8 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   if (p->dtype != PQHSA_F16 && p->dtype != PQHSA_BF16) return PQHSA_ERR_INVALID_ARG;
   if (!(p->sm_scale > 0.f)) return PQHSA_ERR_INVALID_ARG;
   if (p->variant < PQHSA_VARIANT_B || p->variant > PQHSA_VARIANT_C2B) return PQHSA_ERR_INVALID_ARG;
-  if (p->table_precision != PQHSA_TABLES_FP32 && p->table_precision != PQHSA_TABLES_FP16)
+  if (p->table_precision != PQHSA_TABLES_FP32 && p->table_precision != PQHSA_TABLES_FP16 &&
+      p->table_precision != PQHSA_TABLES_FP16_RESCORE)
     return PQHSA_ERR_INVALID_ARG;
   if ((long long)p->max_pages_per_seq * p->page_size < p->max_seq_len) return PQHSA_ERR_INVALID_ARG;
   long long k_need = ((long long)p->max_seq_len * p->budget_ppm + 999999LL) / 1000000LL;
@@ -70,7 +71,7 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   const int G = p->n_q_heads / p->n_kv_heads;
   if (G > 16) return PQHSA_ERR_UNSUPPORTED;
   // fp16 tables: the layer shape of the benchmark only (32 one-byte subspaces, groups of 4 heads)
-  if (p->table_precision == PQHSA_TABLES_FP16 && (p->pq_ncode != 256 || p->pq_m != 32 || G < 3))
+  if (p->table_precision != PQHSA_TABLES_FP32 && (p->pq_ncode != 256 || p->pq_m != 32 || G < 3))
     return PQHSA_ERR_UNSUPPORTED;
 
   Plan& o = *pl;
@@ -83,7 +84,9 @@ int make_plan(const pqhsa_params* p, Plan* pl) {
   o.k_max = p->k_max; o.n_sink = p->n_sink; o.n_local = p->n_local;
   o.exact_multiple = p->exact_set_multiple; o.ppm = p->budget_ppm; o.sm_scale = p->sm_scale; o.dtype = p->dtype;
   o.variant = p->variant; o.indexed_lens = p->indexed_lens; o.status = nullptr;
-  o.half_tables = p->table_precision == PQHSA_TABLES_FP16 ? 1 : 0;
+  o.half_tables = p->table_precision != PQHSA_TABLES_FP32 ? 1 : 0;
+  o.rescore = p->table_precision == PQHSA_TABLES_FP16_RESCORE ? 1 : 0;
+  o.norm_seg = nullptr;
   o.num_sms = sm_count();
   o.scan_ctas = o.num_sms;                                  // persistent scan CTAs: one per SM
   o.upb = o.Hkv * o.n_hg;
@@ -185,6 +188,7 @@ void make_layout(const Plan& pl, WsLayout* L) {
   L->cand = take((size_t)pl.rows * pl.cand_cap * 8);
   L->bg_max = take((size_t)pl.rows * 4);
   L->split_part = take((size_t)pl.rows * attend_parts(pl) * (4 + kHeadDim) * 4);
+  L->norm_seg = take(pl.half_tables ? (size_t)pl.B * pl.upb * pl.n_part * 4 : 0);
   L->stage_end = o;
   L->lut = take(buffer_elems(pl, PQHSA_BUF_LUT) * 4);
   L->coarse = take(buffer_elems(pl, PQHSA_BUF_COARSE) * 4);
@@ -291,8 +295,8 @@ int pqhsa_decode_launch_count(const pqhsa_params* params) {
   int rc = make_plan(params, &pl);
   if (rc != PQHSA_OK) return rc;
   // LUT build, scan, select sample, select filter, background preparation, attend (+ the
-  // correction pass of variant Bx)
-  return pl.variant == PQHSA_VARIANT_BX ? 7 : 6;
+  // correction pass of variant Bx, + the re-score pass of the fp16 tables)
+  return 6 + (pl.variant == PQHSA_VARIANT_BX ? 1 : 0) + (pl.rescore ? 1 : 0);
 }
 
 int pqhsa_build_lut(const pqhsa_params* params, const void* q, const pqhsa_index* index,
@@ -321,6 +325,7 @@ int pqhsa_scan(const pqhsa_params* params, const pqhsa_index* index, const float
   make_layout(pl, &L);
   if ((rc = check_ws(ws, ws_bytes, L.stage_end)) != PQHSA_OK) return rc;
   char* w = static_cast<char*>(ws);
+  if (pl.half_tables) pl.norm_seg = reinterpret_cast<float*>(w + L.norm_seg);
   return cuda_status(launch_scan(pl, *index, lut, coarse, seq_lens, scores, list_partials,
                                  reinterpret_cast<int*>(w + L.status),
                                  static_cast<cudaStream_t>(stream)));
@@ -342,6 +347,26 @@ int pqhsa_select(const pqhsa_params* params, const float* scores, const int32_t*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(w + L.zero_begin, 0, L.zero_bytes, st) != cudaSuccess) return PQHSA_ERR_CUDA;
   return cuda_status(launch_select(pl, L, w, scores, seq_lens, sel_idx, sel_count, kth_score, st));
+}
+
+int pqhsa_rescore(const pqhsa_params* params, const pqhsa_index* index, const float* lut,
+                  const float* coarse, const float* scores, const int32_t* seq_lens,
+                  int32_t* sel_idx, const int32_t* sel_count, float* kth_score, void* ws,
+                  size_t ws_bytes, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if (!pl.rescore) return PQHSA_ERR_INVALID_ARG;
+  if ((rc = check_index(index)) != PQHSA_OK) return rc;
+  if (lut == nullptr || coarse == nullptr || scores == nullptr || seq_lens == nullptr ||
+      sel_idx == nullptr || sel_count == nullptr || kth_score == nullptr)
+    return PQHSA_ERR_INVALID_ARG;
+  WsLayout L;
+  make_layout(pl, &L);
+  if ((rc = check_ws(ws, ws_bytes, L.stage_end)) != PQHSA_OK) return rc;
+  return cuda_status(launch_rescore(pl, L, static_cast<char*>(ws), *index, lut, coarse, scores,
+                                    seq_lens, sel_idx, sel_count, kth_score,
+                                    static_cast<cudaStream_t>(stream)));
 }
 
 int pqhsa_hybrid_attend(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
@@ -399,11 +424,14 @@ static int decode_impl(const pqhsa_params* params, const void* q, const pqhsa_in
   if (e == cudaSuccess)
     e = launch_build_lut(pl, q, *index, lut, coarse, w + L.zero_begin, L.zero_bytes, st);
   if (e == cudaSuccess) e = mark(1);
+  if (pl.half_tables) pl.norm_seg = reinterpret_cast<float*>(w + L.norm_seg);
   if (e == cudaSuccess)
     e = launch_scan(pl, *index, lut, coarse, seq_lens, scores, partials,
                     reinterpret_cast<int*>(w + L.status), st);
   if (e == cudaSuccess) e = mark(2);
   if (e == cudaSuccess) e = launch_select(pl, L, w, scores, seq_lens, sel_idx, sel_count, kth, st);
+  if (e == cudaSuccess && pl.rescore)
+    e = launch_rescore(pl, L, w, *index, lut, coarse, scores, seq_lens, sel_idx, sel_count, kth, st);
   if (e == cudaSuccess) e = mark(3);
   if (e == cudaSuccess)
     e = launch_attend(pl, L, w, q, *kv, *index, scores, partials, sel_idx, sel_count, seq_lens,

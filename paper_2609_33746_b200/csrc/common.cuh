@@ -36,6 +36,8 @@ struct Plan {
   int exact_multiple;                // > 1: |S| + |L| + k is rounded up to this multiple (App. A)
   int variant;                       // pqhsa_variant: how the background term is formed
   int half_tables;                   // scan keeps its lookup tables in fp16 (approximate scores)
+  int rescore;                       // ... and the top-k is re-decided from fp32 tables near its threshold
+  float* norm_seg;                   // device [units][n_part]: largest key norm per scan segment (fp16 tables), or null
   const int32_t* indexed_lens;       // device [B] or null: positions covered by the index
   int* status;                       // device status word, or null (set by the launchers)
   uint32_t ppm;
@@ -70,6 +72,7 @@ struct WsLayout {
   size_t bg_tcount;                  // int32  [rows][n_list]: selected tokens per list (variant Bx only)
   size_t bg_max;                     // float  [rows]
   size_t split_part;                 // float  [rows][splits + bg_splits][4 + 128]: m, Z, pad, N[128]
+  size_t norm_seg;                   // float  [units][n_part]: largest key norm per scan segment (fp16 tables)
   size_t stage_end;                  // end of what a single stage call needs
   // intermediates of the fused entry point
   size_t lut, coarse, scores, list_partials, sel_idx, sel_count, kth;
@@ -90,6 +93,7 @@ int attend_parts(const Plan& plan);                        // partials per score
 constexpr int kStatusCountMismatch = 1;    // top-k emitted a number of positions other than k
 constexpr int kStatusSeqLen = 2;           // seq_lens[b] outside [0, max_seq_len]
 constexpr int kStatusCopyTimeout = 4;      // a bounded wait on a bulk copy ran out
+constexpr int kStatusRescoreSkipped = 64;  // fp16 tables: a row's near-threshold pool did not fit; its top-k is the approximate one
 constexpr int kStatusListId = 8;           // debug: list id >= n_list
 constexpr int kStatusPosition = 16;        // debug: selected position outside the indexed region
 constexpr int kStatusPage = 32;            // debug: negative page id in the block table
@@ -264,6 +268,12 @@ cudaError_t launch_build_lut(const Plan& pl, const void* q, const pqhsa_index& i
 cudaError_t launch_scan(const Plan& pl, const pqhsa_index& ix, const float* lut,
                         const float* coarse, const int32_t* seq_lens, float* scores,
                         float* list_partials, int* status, cudaStream_t st);
+// fp16 tables with re-score: re-decides every row's top-k among the tokens whose approximate
+// score is within the table-rounding bound of the k-th one, from the fp32 tables.
+cudaError_t launch_rescore(const Plan& pl, const WsLayout& L, char* ws, const pqhsa_index& ix,
+                           const float* lut, const float* coarse, const float* scores,
+                           const int32_t* seq_lens, int32_t* sel_idx, const int32_t* sel_count,
+                           float* kth, cudaStream_t st);
 cudaError_t launch_select(const Plan& pl, const WsLayout& L, char* ws, const float* scores,
                           const int32_t* seq_lens, int32_t* sel_idx, int32_t* sel_count,
                           float* kth, cudaStream_t st);

@@ -208,6 +208,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
     ++b;
   }
 
+  [[maybe_unused]] float nmax = 0.f;     // fp16 tables: largest key norm seen in the segment
   while (lo < hi && b < pl.B) {
     const int tb = seq_tiles(seq_lens, b, N_max);
     const int w = (int)((lo - base) / tb);
@@ -295,6 +296,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
       const int i = t * kTile + lane;
       const bool valid = have && i < Nb;
       const bool in_r = valid && i >= rg.r_begin && i < rg.r_end;
+      if constexpr (kHalf) nmax = fmaxf(nmax, cur.norm);
       float sc[GC];
 #pragma unroll
       for (int g = 0; g < GC; ++g) sc[g] = -CUDART_INF_F;
@@ -473,6 +475,20 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
         }
         if (any) red_add<GC>(part_sums + (size_t)lid * GC, e);
       }
+    }
+    if constexpr (kHalf) {
+      // largest key norm of the segment: with it the re-score pass bounds the error that the
+      // fp16 tables put on any score of the row
+      const float v = warp_max(nmax);
+      __syncthreads();
+      if (lane == 0) s_red[warp][0] = v;
+      __syncthreads();
+      if (tid == 0 && pl.norm_seg != nullptr) {
+        float m = 0.f;
+        for (int ww = 0; ww < kWarps; ++ww) m = fmaxf(m, s_red[ww][0]);
+        pl.norm_seg[unit * pl.n_part + slot] = m;
+      }
+      nmax = 0.f;
     }
     // header: the reference the sums are relative to (same units as the scores; the exponent
     // was formed as fma(l~, log2 e, -(ref * log2 e)) in base 2) and the segment's maximum; a

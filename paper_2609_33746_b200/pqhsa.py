@@ -32,6 +32,7 @@ EXPORTS = [
     "pqhsa_select_static_bytes", "pqhsa_select_static_capacity", "pqhsa_dense_decode",
     "pqhsa_dense_workspace_bytes", "pqhsa_index_update", "pqhsa_debug_build",
     "pqhsa_debug_predicate", "pqhsa_index_build", "pqhsa_index_build_workspace_bytes",
+    "pqhsa_rescore",
 ]
 
 
@@ -93,6 +94,7 @@ def lib() -> ctypes.CDLL:
             "pqhsa_build_lut": (I, [P, V, PI, V, V, V]),
             "pqhsa_scan": (I, [P, PI, V, V, V, V, V, V, Z, V]),
             "pqhsa_select": (I, [P, V, V, V, V, V, V, Z, V]),
+            "pqhsa_rescore": (I, [P, PI, V, V, V, V, V, V, V, V, Z, V]),
             "pqhsa_hybrid_attend": (I, [P, V, PK, PI, V, V, V, V, V, V, V, V, V, Z, V]),
             "pqhsa_decode": (I, [P, V, PI, PK, V, V, V, Z, V]),
             "pqhsa_decode_events": (I, [P, V, PI, PK, V, V, V, Z, V, ctypes.POINTER(V)]),
@@ -145,7 +147,9 @@ def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_
                 budget_ppm, dtype, head_dim=128, pq_ncode=256, page_size=16, n_sink=0, n_local=0,
                 k_max=None, sm_scale=None, exact_set_multiple=0, variant="B",
                 indexed_lens=None, fp16_tables=False) -> Params:
-    """`indexed_lens`: device int32 tensor [batch] or None; the caller keeps it alive."""
+    """`indexed_lens`: device int32 tensor [batch] or None; the caller keeps it alive.
+    `fp16_tables`: False, True (fp16 tables in the scan) or "rescore" (fp16 tables and the fp32
+    re-score of the top-k's threshold zone)."""
     if k_max is None:
         k_max = max(1, (max_seq_len * budget_ppm + 999_999) // 1_000_000)
         if exact_set_multiple > 1:
@@ -155,7 +159,7 @@ def make_params(*, batch, n_q_heads, n_kv_heads, n_list, pq_m, max_seq_len, max_
     code = {"fp16": F16, "bf16": BF16, torch.float16: F16, torch.bfloat16: BF16}[dtype]
     return Params(batch, n_q_heads, n_kv_heads, head_dim, n_list, pq_m, head_dim // pq_m, pq_ncode,
                   max_seq_len, page_size, max_pages_per_seq, n_sink, n_local, budget_ppm, k_max,
-                  sm_scale, code, exact_set_multiple, VARIANTS[variant], 1 if fp16_tables else 0,
+                  sm_scale, code, exact_set_multiple, VARIANTS[variant], {False: 0, True: 1, "rescore": 2}[fp16_tables],
                   _ptr(indexed_lens))
 
 
@@ -223,6 +227,14 @@ def select(params, scores, seq_lens, sel_idx, sel_count, kth_score, ws, stream=N
     _check("pqhsa_select", lib().pqhsa_select(
         ctypes.byref(params), _ptr(scores), _ptr(seq_lens), _ptr(sel_idx), _ptr(sel_count),
         _ptr(kth_score), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def rescore(params, index, lut, coarse, scores, seq_lens, sel_idx, sel_count, kth_score, ws,
+            stream=None) -> None:
+    _check("pqhsa_rescore", lib().pqhsa_rescore(
+        ctypes.byref(params), ctypes.byref(index), _ptr(lut), _ptr(coarse), _ptr(scores),
+        _ptr(seq_lens), _ptr(sel_idx), _ptr(sel_count), _ptr(kth_score), _ptr(ws),
+        ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def select_static_capacity() -> int:

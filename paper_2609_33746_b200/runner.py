@@ -14,7 +14,7 @@ class DecodeOp:
 
     def __init__(self, inp: DecodeInputs, index: IvfPqIndex, device: str = "cuda:0",
                  budget_ppm: int | None = None, variant: str | None = None,
-                 fp16_tables: bool = False):
+                 fp16_tables=False):
         cfg: DecodeConfig = inp.cfg
         self.cfg, self.device = cfg, torch.device(device)
         dev = self.device
@@ -54,6 +54,7 @@ class DecodeOp:
                                       self.key_norms, self.list_vmeans, self.list_counts)
         self.kv = pqhsa.make_paged_kv(self.k_cache, self.v_cache, inp.stride_page,
                                       inp.stride_token, inp.stride_head, self.block_table)
+        self.fp16_tables = fp16_tables
         self.ws = torch.empty(pqhsa.workspace_bytes(self.params), dtype=torch.uint8, device=dev)
         self.out = torch.zeros_like(self.q)
 
@@ -82,6 +83,9 @@ class DecodeOp:
     def select(self):
         pqhsa.select(self.params, self.scores, self.seq_lens, self.sel_idx, self.sel_count,
                      self.kth, self.ws)
+        if self.fp16_tables == "rescore":
+            pqhsa.rescore(self.params, self.index, self.lut, self.coarse, self.scores, self.seq_lens,
+                          self.sel_idx, self.sel_count, self.kth, self.ws)
 
     def hybrid_attend(self):
         pqhsa.hybrid_attend(self.params, self.q, self.kv, self.index, self.scores,

@@ -1,4 +1,5 @@
-"""The opt-in fp16-table mode of the scan (pqhsa_params.table_precision = PQHSA_TABLES_FP16), -m gpu.
+"""The opt-in fp16-table modes of the scan (pqhsa_params.table_precision = PQHSA_TABLES_FP16 and
+PQHSA_TABLES_FP16_RESCORE), -m gpu.
 
 In this mode the approximate logits carry the rounding of fp16 table entries, so the scan stage is
 NOT held to the 1e-4 logit tolerance.  What is checked instead, against the float64 oracle on the
@@ -20,8 +21,8 @@ from oracle import pqhsa_oracle as O
 from paper_2609_33746_b200 import pqhsa
 from paper_2609_33746_b200.runner import DecodeOp
 
-from helpers import make_case, oracle_arrays, run_oracle
-from test_gpu_parity import OUT_ATOL, small
+from helpers import make_case, oracle_arrays, run_oracle, selection_matches
+from test_gpu_parity import LOGIT_RTOL, OUT_ATOL, out_tolerance, small
 
 pytestmark = pytest.mark.gpu
 
@@ -32,6 +33,10 @@ CASES = {
     "g3_padded_fp16_cache": small("h_g3", n_q_heads=6, n_kv_heads=2, seq_lens=(2777,), dtype="fp16"),
     "many_lists": small("h_l", seq_lens=(6000,), n_list=1024, n_q_heads=4, n_kv_heads=1, kmeans_iters=2),
 }
+FP32_TIE = 2e-5     # two scores this close (relative to max(1, |s_k|)) may swap between fp32 and fp64
+# long enough for the threshold zone to hold tokens that the fp16 tables rank differently
+LONG = small("h_long", seq_lens=(60000, 41000), batch=2, n_q_heads=8, n_kv_heads=2, n_list=256,
+             budget_ppm=20000, kmeans_iters=1)
 
 
 @pytest.mark.parametrize("key", list(CASES))
@@ -97,6 +102,105 @@ def test_fp16_tables_scores_selection_and_output(key):
         assert np.abs(y32[b, h] - y_dev_sel).max() <= OUT_ATOL
         assert np.abs(y32[b, h] - r["y"]).max() <= 5 * OUT_ATOL     # and near the fp32-table result
     assert worst_ratio <= 1.0 and np.mean(mean_err) > 1e-6          # approximate, inside its bound
+
+
+@pytest.mark.parametrize("key", list(CASES) + ["long"])
+def test_fp16_tables_with_rescore_select_what_fp32_tables_select(key):
+    """With the fp32 re-score of the threshold zone the selected set is the oracle's up to ties at
+    the level of fp32 rounding (2e-5 relative, far below the fp16 tables' error), the k-th score is
+    the fp32 one, and the output meets the usual tolerance against the oracle's output; the fused
+    call gives the staged calls' result."""
+    cfg = LONG if key == "long" else CASES[key]
+    inp, idx = make_case(cfg, device="cuda")
+    arrays = oracle_arrays(inp, idx)
+    ref = run_oracle(inp, idx, arrays=arrays)
+    plain = DecodeOp(inp, idx, fp16_tables=True)
+    plain.alloc_stage_buffers()
+    plain.build_lut(); plain.scan(); plain.select()
+    op = DecodeOp(inp, idx, fp16_tables="rescore")
+    op.alloc_stage_buffers()
+    op.build_lut(); op.scan()
+    op.sel_idx.fill_(-1)
+    op.select()                                   # top-k on the fp16-table scores, then the re-score
+    op.out_f32.fill_(5.0)
+    op.hybrid_attend()
+    torch.cuda.synchronize()
+    assert op.device_status() == pqhsa.OK
+    assert pqhsa.decode_launch_count(op.params) == pqhsa.decode_launch_count(plain.params) + 1
+    k_max = op.params.k_max
+    sel = op.sel_idx.view(cfg.batch, cfg.n_q_heads, k_max).cpu().numpy()
+    sel_plain = plain.sel_idx.view(cfg.batch, cfg.n_q_heads, k_max).cpu().numpy()
+    cnt = op.sel_count.view(cfg.batch, cfg.n_q_heads).cpu().numpy()
+    kth = op.kth.view(cfg.batch, cfg.n_q_heads).cpu().numpy()
+    y32 = op.out_f32.cpu().double().numpy()
+    moved, plain_off = 0, 0
+    for (b, h), r in ref.items():
+        k = r["k"]
+        assert cnt[b, h] == k
+        ok, why = selection_matches(sel[b, h, :k], r, tol=FP32_TIE)
+        assert ok, f"{(b, h)}: {why}"
+        moved += len(set(sel[b, h, :k].tolist()) ^ set(sel_plain[b, h, :k].tolist()))
+        plain_off += 0 if selection_matches(sel_plain[b, h, :k], r, tol=FP32_TIE)[0] else 1
+        if k:
+            assert abs(kth[b, h] - r["kth_score"]) <= LOGIT_RTOL * max(1.0, abs(r["kth_score"]))
+        assert np.abs(y32[b, h] - r["y"]).max() <= OUT_ATOL
+    print(f"{key}: the re-score moved {moved} positions; rows where the fp16 tables alone miss: {plain_off}")
+    if key == "long":
+        assert moved > 0 and plain_off > 0        # the case does exercise the re-score
+    op.out.zero_()
+    op.decode()
+    torch.cuda.synchronize()
+    assert op.device_status() == pqhsa.OK
+    fused_sel = op.decode_buffer(pqhsa.BUF_SEL_IDX, torch.int32).view(cfg.batch, cfg.n_q_heads, k_max).cpu().numpy()
+    for (b, h), r in ref.items():
+        assert sorted(fused_sel[b, h, :r["k"]].tolist()) == sorted(sel[b, h, :r["k"]].tolist())
+    fused = op.out.cpu().double().numpy()
+    for (b, h), r in ref.items():
+        assert np.all(np.abs(fused[b, h] - r["y"]) <= out_tolerance(r["y"], cfg.dtype))
+
+
+@pytest.mark.parametrize("factor,expect_skip", [(20.0, False), (3000.0, True)])
+def test_rescore_with_one_huge_key_norm(factor, expect_skip):
+    """The error bound of a row scales with the largest key norm in it.  One token with a norm 20
+    times the others' widens every row's threshold zone twentyfold and the re-score still lands on
+    the oracle's set; a norm 3000 times larger makes the zone wider than the pool the kernel can
+    hold, and the rows then KEEP the exact top-k of the fp16-table scores and say so in the status
+    word (bit 64) -- nothing is dropped or duplicated."""
+    cfg = small("h_norm", seq_lens=(30000,), n_q_heads=4, n_kv_heads=1, n_list=256,
+                budget_ppm=20000, kmeans_iters=1)
+    inp, idx = make_case(cfg, device="cuda")
+    idx.key_norms[0, 0, 777] *= factor
+    arrays = oracle_arrays(inp, idx)
+    ref = run_oracle(inp, idx, arrays=arrays)
+    op = DecodeOp(inp, idx, fp16_tables="rescore")
+    op.alloc_stage_buffers()
+    op.build_lut(); op.scan(); op.select()
+    torch.cuda.synchronize()
+    k_max = op.params.k_max
+    sel = op.sel_idx.view(cfg.batch, cfg.n_q_heads, k_max).cpu().numpy()
+    scores = op.scores.view(cfg.batch, cfg.n_q_heads, -1).cpu().double().numpy()
+    if expect_skip:
+        assert op.device_status() == pqhsa.ERR_DEVICE_CHECK
+        for (b, h), r in ref.items():
+            r0, r1 = int(r["R"][0]), int(r["R"][-1]) + 1
+            want = (O.select_topk(scores[b, h, r0:r1], r["k"]) + r0).tolist()
+            assert sorted(sel[b, h, :r["k"]].tolist()) == want
+    else:
+        assert op.device_status() == pqhsa.OK
+        for (b, h), r in ref.items():
+            ok, why = selection_matches(sel[b, h, :r["k"]], r, tol=FP32_TIE)
+            assert ok, f"{(b, h)}: {why}"
+
+
+def test_rescore_entry_point_is_refused_without_the_mode():
+    cfg = small("h_plain", seq_lens=(1000,))
+    inp, idx = make_case(cfg, device="cuda")
+    op = DecodeOp(inp, idx, fp16_tables=True)
+    op.alloc_stage_buffers()
+    with pytest.raises(pqhsa.PqhsaError) as e:
+        pqhsa.rescore(op.params, op.index, op.lut, op.coarse, op.scores, op.seq_lens, op.sel_idx,
+                      op.sel_count, op.kth, op.ws)
+    assert e.value.status == pqhsa.ERR_INVALID_ARG
 
 
 def test_fp16_tables_are_refused_outside_the_supported_shape():

@@ -326,14 +326,16 @@ def test_many_candidates_take_the_global_list_path():
         assert sorted(got[h, :k].tolist()) == want.tolist()
 
 
-def sampled_positions(n, n_groups=1024):
-    """The positions the select's sample kernel reads in a row of n scores (1024 groups of 4)."""
-    g = np.arange(n_groups, dtype=np.int64)
-    a, z = g * n // n_groups, (g + 1) * n // n_groups
-    h = (g * 2654435761) & 0xFFFFFFFF
-    off = (a + (h >> 8) % (z - a)) & ~3
-    off = np.where(off + 4 > n, (n - 4) & ~3, off)
-    return (off[:, None] + np.arange(4)[None, :]).ravel()
+def sampled_positions(n):
+    """The positions the select's sample kernel reads in a row of n scores (groups of 16 scores at
+    a hashed offset inside equal strides; at most 1024 groups and a quarter of the row)."""
+    n_groups = min(1024, n // 64)
+    stride = n // n_groups
+    g = np.arange(n_groups, dtype=np.uint64)
+    h = (g * np.uint64(2654435761)) & np.uint64(0xFFFFFFFF)
+    off = (g * np.uint64(stride) + ((h * np.uint64(stride)) >> np.uint64(32))) & ~np.uint64(15)
+    off = np.minimum(off, np.uint64((n - 16) & ~15)).astype(np.int64)
+    return (off[:, None] + np.arange(16)[None, :]).ravel()
 
 
 def test_rows_that_defeat_the_sample_fall_back_to_the_exact_path():

@@ -359,6 +359,39 @@ def main():
         table_wavefronts_per_tile=(cfg.pq_m if cfg.pq_ncode > 16 else cfg.pq_m) * 4,
         tiles_per_launch=scan_tiles)
 
+    # the attend stage against the memory system's price for its gather: a probe that reads the
+    # selected tokens' K and V rows (same addresses, through the block table) and computes
+    # nothing, timed like a stage (after the L2 flush, whose dirty lines the kernel that follows
+    # has to write back) and once more behind a read sweep that leaves L2 clean
+    sel_idx = op.decode_buffer(pqhsa.BUF_SEL_IDX, torch.int32)
+    sel_count = op.decode_buffer(pqhsa.BUF_SEL_COUNT, torch.int32)
+    sink = torch.zeros(4, dtype=torch.int32, device=dev)
+    sweep_src = torch.empty(256 << 20, dtype=torch.uint8, device=dev).zero_()
+
+    def probe_us(after_flush):
+        ts = []
+        for _ in range(12):
+            if after_flush:
+                flush.zero_()
+            else:
+                flush.zero_()
+                sweep_src.sum()                       # reads 256 MB: what L2 holds afterwards is clean
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            pqhsa.gather_probe(op.params, op.kv, sel_idx, sel_count, op.seq_lens, sink)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(1000 * a.elapsed_time(b))
+        return statistics.median(ts[2:])
+    gather_bytes = int(sel_count.sum().item()) * 2 * cfg.head_dim * 2      # a K and a V row per selected token
+    pu_dirty, pu_clean = probe_us(True), probe_us(False)
+    roofline["attend_gather_probe"] = dict(
+        what="pqhsa_gather_probe: the selected K/V rows read through the block table, nothing computed",
+        bytes=gather_bytes, us_after_dirty_l2_flush=pu_dirty, us_after_clean_l2=pu_clean,
+        gbs_after_dirty_l2_flush=gather_bytes / pu_dirty / 1e3, gbs_after_clean_l2=gather_bytes / pu_clean / 1e3,
+        attend_stage_us=1000 * stage_ms[3])
+    del sweep_src
+
     # end to end through the host-buffer entry point: q from pinned host memory, out back
     q_host = op.q.cpu().pin_memory()
     out_host = torch.empty_like(q_host).pin_memory()

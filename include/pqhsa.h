@@ -338,6 +338,15 @@ size_t pqhsa_dense_workspace_bytes(const pqhsa_params* params);
 int pqhsa_dense_decode(const pqhsa_params* params, const void* q, const pqhsa_paged_kv* kv,
                        const int32_t* seq_lens, void* out, void* ws, size_t ws_bytes, void* stream);
 
+/* Measurement aid, not a step of the method: reads the K and V rows of the selected tokens (the
+ * addresses the exact part of pqhsa_hybrid_attend gathers, through the same block table and
+ * strides) with many rows in flight and computes nothing.  Its duration is the memory system's
+ * price for that gather, the ceiling the attend stage is set against in the benchmark.
+ * sel_idx / sel_count as pqhsa_select leaves them; sink16: 16 device bytes, 16-byte aligned,
+ * never written in practice.  One launch on `stream`. */
+int pqhsa_gather_probe(const pqhsa_params* params, const pqhsa_paged_kv* kv, const int32_t* sel_idx,
+                       const int32_t* sel_count, const int32_t* seq_lens, void* sink16, void* stream);
+
 /* pqhsa_decode for a caller whose query and output live in HOST memory (pinned for the
  * copies to be asynchronous): copies q_host -> q_dev_staging, runs the step, copies
  * out_dev_staging -> out_host and waits for the stream.  The index, the KV cache and

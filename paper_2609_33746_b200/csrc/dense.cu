@@ -184,6 +184,62 @@ int dense_splits(const Plan& pl) {
 
 size_t align256d(size_t x) { return (x + 255) / 256 * 256; }
 
+// Read-only probe of the gather that the exact part of the attend step performs: the K and V
+// rows of the selected tokens, through the block table and the strides, nothing computed (the
+// words are xor-ed into a sink that is never written).  A warp takes 32 selected tokens of a
+// row at a time: every lane resolves one token's address (position, page) one round ahead,
+// then half-warps fetch the K and the V rows, sixteen tokens in flight.  Its time is what the
+// memory system charges for these bytes at these addresses: the ceiling the attend kernel is
+// measured against.
+constexpr int kProbeRows = 16;      // selected tokens per warp in flight (K and V row each)
+
+__global__ void __launch_bounds__(256)
+gather_probe_kernel(Plan pl, const unsigned char* __restrict__ kc, const unsigned char* __restrict__ vc,
+                    long long stride_page, long long stride_token, long long stride_head,
+                    const int32_t* __restrict__ block_table, const int32_t* __restrict__ sel_idx,
+                    const int32_t* __restrict__ sel_count, const int32_t* __restrict__ seq_lens,
+                    uint4* __restrict__ sink) {
+  const int lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+  const int warp = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  const int n_warps = (int)((gridDim.x * blockDim.x) >> 5);
+  const int cpr = (pl.k_max + 31) / 32;                  // rounds of 32 tokens per row
+  const int rounds = pl.rows * cpr;
+  const unsigned char* base = half ? vc : kc;            // lanes 0-15: the K row, 16-31: the V row
+  uint4 acc = make_uint4(0u, 0u, 0u, 0u);
+  // byte offset of the row of this lane's token in round r, -1 if there is none
+  auto resolve = [&](int r) -> long long {
+    if (r >= rounds) return -1;
+    const int row = r / cpr, t = (r - row * cpr) * 32 + lane;
+    const int b = row / pl.Hq, kv = (row % pl.Hq) / pl.G;
+    const int cnt = min(max(__ldg(sel_count + row), 0), pl.k_max);
+    if (t >= cnt) return -1;
+    const int pos = __ldg(sel_idx + (size_t)row * pl.k_max + t);
+    if ((unsigned)pos >= (unsigned)clamp_len(seq_lens[b], pl.N_max)) return -1;
+    const int page = __ldg(block_table + (size_t)b * pl.max_pages + pos / pl.page_size);
+    return 2 * ((long long)page * stride_page + (long long)(pos % pl.page_size) * stride_token +
+                (long long)kv * stride_head);             // strides are in 2-byte elements
+  };
+  long long off = resolve(warp);
+  for (int r = warp; r < rounds; r += n_warps) {
+    const long long nxt = resolve(r + n_warps);
+#pragma unroll
+    for (int j0 = 0; j0 < 32; j0 += kProbeRows) {
+      uint4 v[kProbeRows];
+#pragma unroll
+      for (int u = 0; u < kProbeRows; ++u) {
+        const long long o = __shfl_sync(0xffffffffu, off, j0 + u);
+        v[u] = o >= 0 ? __ldg(reinterpret_cast<const uint4*>(base + o) + l16) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int u = 0; u < kProbeRows; ++u) { acc.x ^= v[u].x; acc.y ^= v[u].y; acc.z ^= v[u].z; acc.w ^= v[u].w; }
+    }
+    off = nxt;
+  }
+  // (the store keeps the loads alive; the pattern does not occur)
+  if (acc.x == 0x9e3779b9u && acc.y == 0x7f4a7c15u && acc.z == 0xf39cc060u && acc.w == 0x5cedc834u)
+    sink[0] = acc;
+}
+
 }  // namespace
 }  // namespace pqhsa
 
@@ -231,6 +287,24 @@ int pqhsa_dense_decode(const pqhsa_params* params, const void* q, const pqhsa_pa
                    static_cast<const __nv_bfloat16*>(kv->v_cache), (long long)kv->stride_page,
                    (long long)kv->stride_token, (long long)kv->stride_head, kv->block_table,
                    seq_lens, part, tickets, static_cast<__nv_bfloat16*>(out));
+  return e == cudaSuccess ? PQHSA_OK : PQHSA_ERR_CUDA;
+}
+
+int pqhsa_gather_probe(const pqhsa_params* params, const pqhsa_paged_kv* kv, const int32_t* sel_idx,
+                       const int32_t* sel_count, const int32_t* seq_lens, void* sink16, void* stream) {
+  Plan pl;
+  int rc = make_plan(params, &pl);
+  if (rc != PQHSA_OK) return rc;
+  if (kv == nullptr || kv->k_cache == nullptr || kv->v_cache == nullptr || kv->block_table == nullptr ||
+      sel_idx == nullptr || sel_count == nullptr || seq_lens == nullptr || sink16 == nullptr ||
+      (reinterpret_cast<uintptr_t>(sink16) & 15u) != 0)
+    return PQHSA_ERR_INVALID_ARG;
+  if (kv->stride_page % 8 || kv->stride_token % 8 || kv->stride_head % 8) return PQHSA_ERR_UNSUPPORTED;
+  const cudaError_t e = launch_pdl(
+      gather_probe_kernel, dim3(8 * pl.num_sms), dim3(256), 0, static_cast<cudaStream_t>(stream), pl,
+      static_cast<const unsigned char*>(kv->k_cache), static_cast<const unsigned char*>(kv->v_cache),
+      (long long)kv->stride_page, (long long)kv->stride_token, (long long)kv->stride_head,
+      kv->block_table, sel_idx, sel_count, seq_lens, static_cast<uint4*>(sink16));
   return e == cudaSuccess ? PQHSA_OK : PQHSA_ERR_CUDA;
 }
 

@@ -32,7 +32,7 @@ EXPORTS = [
     "pqhsa_select_static_bytes", "pqhsa_select_static_capacity", "pqhsa_dense_decode",
     "pqhsa_dense_workspace_bytes", "pqhsa_index_update", "pqhsa_debug_build",
     "pqhsa_debug_predicate", "pqhsa_index_build", "pqhsa_index_build_workspace_bytes",
-    "pqhsa_rescore",
+    "pqhsa_rescore", "pqhsa_gather_probe",
 ]
 
 
@@ -108,6 +108,7 @@ def lib() -> ctypes.CDLL:
             "pqhsa_select_static_capacity": (Z, []),
             "pqhsa_dense_decode": (I, [P, V, PK, V, V, V, Z, V]),
             "pqhsa_dense_workspace_bytes": (Z, [P]),
+            "pqhsa_gather_probe": (I, [P, PK, V, V, V, V, V]),
             "pqhsa_index_update": (I, [P, ctypes.POINTER(IndexRW), PK, V, V, I, V]),
             "pqhsa_index_build_workspace_bytes": (Z, [P]),
             "pqhsa_index_build": (I, [P, PK, V, V, V, I, I, ctypes.POINTER(IndexOut), V, Z, V]),
@@ -235,6 +236,13 @@ def rescore(params, index, lut, coarse, scores, seq_lens, sel_idx, sel_count, kt
         ctypes.byref(params), ctypes.byref(index), _ptr(lut), _ptr(coarse), _ptr(scores),
         _ptr(seq_lens), _ptr(sel_idx), _ptr(sel_count), _ptr(kth_score), _ptr(ws),
         ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def gather_probe(params, kv: PagedKV, sel_idx, sel_count, seq_lens, sink, stream=None) -> None:
+    """Measurement aid: reads the selected tokens' K and V rows and computes nothing."""
+    _check("pqhsa_gather_probe", lib().pqhsa_gather_probe(
+        ctypes.byref(params), ctypes.byref(kv), _ptr(sel_idx), _ptr(sel_count), _ptr(seq_lens),
+        _ptr(sink), _stream(stream)))
 
 
 def select_static_capacity() -> int:

@@ -447,6 +447,16 @@ def test_dense_comparator_is_textbook_attention(key):
             assert np.all(np.abs(got[b, h] - want) <= out_tolerance(want, cfg.dtype))
 
 
+def test_gather_probe_runs_and_writes_nothing():
+    """The measurement aid reads the selected rows and leaves its sink alone."""
+    inp, idx, arrays, ref, op = get_case(next(iter(CASES)))
+    op.build_lut(); op.scan(); op.select()
+    sink = torch.zeros(4, dtype=torch.int32, device="cuda")
+    pqhsa.gather_probe(op.params, op.kv, op.sel_idx, op.sel_count, op.seq_lens, sink)
+    torch.cuda.synchronize()
+    assert int(sink.abs().sum()) == 0 and op.device_status() == pqhsa.OK
+
+
 def test_paper_budgets_on_the_device():
     """App. A prints the exact-set sizes of the 128K setting (4 sinks, 128-token window, pages
     of 16): the device's integer budget arithmetic must land on the same totals, and the

@@ -53,6 +53,8 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = pl.G, Gc = pl.Gc, n_hg = pl.n_hg;
   const int n_slots = n_hg * Gc;                            // head slots, >= G
+  const int gc_shift = Gc == 4 ? 2 : (Gc == 2 ? 1 : 0);     // Gc is 1, 2 or 4
+  const int code_shift = 31 - __clz(pl.n_code);             // n_code is 16 or 256
   const size_t ukv = (size_t)b * pl.Hkv + kv;
   pdl_wait();
   pdl_launch_dependents();
@@ -126,46 +128,62 @@ build_lut_kernel(Plan pl, const T* __restrict__ q, const float* __restrict__ cen
           crow[u] = __ldg(reinterpret_cast<const float4*>(centroids + (ukv * pl.n_list + j) * kHeadDim) + lane);
       }
     }
+    // the lane's slice of the four query heads is the same for every row: one set of reads per
+    // batch of rows
+    for (int hb = 0; hb < n_slots; hb += 4) {
+      float4 qq[4];
 #pragma unroll
-    for (int u = 0; u < kRowsPerWarp; ++u) {
-      const int j = jb + warp + u * kLutWarps;
-      if (j >= r1) continue;                       // warp-uniform
-      const float4 c = crow[u];
-      for (int hb = 0; hb < n_slots; hb += 4) {
+      for (int t = 0; t < 4; ++t)
+        qq[t] = *reinterpret_cast<const float4*>(&sq[(hb + t) & (kMaxGroup - 1)][4 * lane]);
+      const int slot = hb + (lane >> 3);
+      const int hg = slot >> gc_shift, g = slot & (Gc - 1);
+      float* dst = coarse + ((ukv * n_hg + hg) * (size_t)pl.n_list) * Gc + g;
+#pragma unroll
+      for (int u = 0; u < kRowsPerWarp; ++u) {
+        const int j = jb + warp + u * kLutWarps;
+        if (j >= r1) continue;                       // warp-uniform
+        const float4 c = crow[u];
         float p[4];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const float4 qq = *reinterpret_cast<const float4*>(&sq[(hb + t) & (kMaxGroup - 1)][4 * lane]);
-          p[t] = c.x * qq.x + c.y * qq.y + c.z * qq.z + c.w * qq.w;
-        }
+        for (int t = 0; t < 4; ++t)
+          p[t] = c.x * qq[t].x + c.y * qq[t].y + c.z * qq[t].z + c.w * qq[t].w;
         const float tot = warp_sum4(p[0], p[1], p[2], p[3], lane);
-        const int slot = hb + (lane >> 3);
-        if ((lane & 7) == 0 && slot < n_slots) {
-          const int hg = slot / Gc, g = slot % Gc;
-          coarse[(((ukv * n_hg + hg) * pl.n_list) + j) * Gc + g] = tot;
-        }
+        if ((lane & 7) == 0 && slot < n_slots) dst[(size_t)j * Gc] = tot;
       }
     }
   }
 
   // ---- PQ table: one thread per (m, z); consecutive threads take consecutive z, so the
   //      subspace m (and with it the query sub-vector) is uniform over a warp
+  float* const lut_u = lut + ukv * n_hg * (size_t)pl.n_code * pl.M * Gc;
   for (int eb = e0; eb < e1; eb += kLutThreads) {
     const int e = eb + tid;
     if (eb != e0 && e < e1) load_codeword(e);
     if (e >= e1) continue;
-    const int m = e / kEntPerM, z = e % kEntPerM;
+    const int m = e >> code_shift, z = e & (kEntPerM - 1);
     for (int hg = 0; hg < n_hg; ++hg) {
       float v[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         if (g < Gc) {
+          // (same products in the same order as a scalar loop; the reads are 8 or 16 bytes wide)
           const float* qs = &sq[(hg * Gc + g) & (kMaxGroup - 1)][m * DSUB];
+          float qv[DSUB];
+          if constexpr (DSUB == 2) {
+            const float2 t2 = *reinterpret_cast<const float2*>(qs);
+            qv[0] = t2.x; qv[1] = t2.y;
+          } else {
 #pragma unroll
-          for (int t = 0; t < DSUB; ++t) v[g] = fmaf(cw[t], qs[t], v[g]);
+            for (int c = 0; c < DSUB / 4; ++c) {
+              const float4 t4 = *reinterpret_cast<const float4*>(qs + 4 * c);
+              qv[4 * c] = t4.x; qv[4 * c + 1] = t4.y; qv[4 * c + 2] = t4.z; qv[4 * c + 3] = t4.w;
+            }
+          }
+#pragma unroll
+          for (int t = 0; t < DSUB; ++t) v[g] = fmaf(cw[t], qv[t], v[g]);
         }
       }
-      float* dst = lut + (((ukv * n_hg + hg) * pl.n_code + z) * pl.M + m) * Gc;
+      float* dst = lut_u + (((size_t)hg * pl.n_code + z) * pl.M + m) * Gc;
       if (Gc == 4) *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
       else if (Gc == 2) *reinterpret_cast<float2*>(dst) = make_float2(v[0], v[1]);
       else dst[0] = v[0];

@@ -392,7 +392,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
       }
 
       if (first) {
-        // reference of the exp-sums: maximum over the first round of tiles of the CTA
+        // reference of the exp-sums: maximum over the first round of tiles of the CTA, plus headroom
 #pragma unroll
         for (int g = 0; g < GC; ++g) {
           const float v = warp_max(mx[g]);
@@ -404,8 +404,9 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
           float v = -CUDART_INF_F;
 #pragma unroll
           for (int ww = 0; ww < kWarps; ++ww) v = fmaxf(v, s_red[ww][g]);
-          ref2[g] = v * kLog2e;
-          if (tid == g) s_ref[g] = v;                    // header value: same units as the scores
+          const float vr = v + kRefHeadroom;            // (-inf stays -inf)
+          ref2[g] = vr * kLog2e;
+          if (tid == g) s_ref[g] = vr;                   // header value: same units as the scores
         }
         first = false;
       }
@@ -419,7 +420,7 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
           xm = fmaxf(xm, x[g]);
         }
         if (xm > kOverflowGuardLog2) s_overflow = 1;
-        if (xm > kNegligibleLog2) {
+        if (xm > kScanNegligibleLog2) {
           float e[GC];
 #pragma unroll
           for (int g = 0; g < GC; ++g) e[g] = fast_exp2(x[g]);
@@ -460,20 +461,32 @@ scan_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restri
       __syncthreads();
       const int i_begin = t0 * kTile;
       const int i_end = min(Nb, tend * kTile);
-      for (int i = i_begin + tid; i < i_end; i += kScanThreads) {
-        const uint32_t lid = min((uint32_t)__ldg(lids + row_base + i), (uint32_t)(n_list - 1));
-        float e[GC];
-        bool any = false;
+      // (eight tokens per thread in flight: the pass is a chain of L2 round trips otherwise)
+      constexpr int kRb = 8;
+      for (int i0 = i_begin + tid; i0 < i_end; i0 += kRb * kScanThreads) {
+        uint32_t lid[kRb];
+        float sv[kRb][GC];
 #pragma unroll
-        for (int g = 0; g < GC; ++g) {
-          e[g] = 0.f;
-          if (g < n_heads) {
-            const float s = __ldcg(scores + (size_t)(row0 + g) * N_max + i);
-            const float x = fmaf(s, kLog2e, -(s_ref[g] * kLog2e));     // -inf outside R
+        for (int u = 0; u < kRb; ++u) {
+          const int i = i0 + u * kScanThreads;
+          lid[u] = i < i_end ? (uint32_t)__ldg(lids + row_base + i) : 0u;
+#pragma unroll
+          for (int g = 0; g < GC; ++g)
+            sv[u][g] = (g < n_heads && i < i_end) ? __ldcg(scores + (size_t)(row0 + g) * N_max + i)
+                                                  : -CUDART_INF_F;
+        }
+#pragma unroll
+        for (int u = 0; u < kRb; ++u) {
+          float e[GC];
+          bool any = false;
+#pragma unroll
+          for (int g = 0; g < GC; ++g) {
+            const float x = fmaf(sv[u][g], kLog2e, -(s_ref[g] * kLog2e));     // -inf outside R
+            e[g] = 0.f;
             if (x > kNegligibleLog2) { e[g] = fast_exp2(x); any = true; }
           }
+          if (any) red_add<GC>(part_sums + (size_t)min(lid[u], (uint32_t)(n_list - 1)) * GC, e);
         }
-        if (any) red_add<GC>(part_sums + (size_t)lid * GC, e);
       }
     }
     if constexpr (kHalf) {

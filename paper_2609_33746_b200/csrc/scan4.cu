@@ -316,7 +316,7 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
       }
 
       if (first) {
-        // reference of the exp-sums: maximum over the first round of the CTA
+        // reference of the exp-sums: maximum over the first round of the CTA, plus headroom
 #pragma unroll
         for (int g = 0; g < GC; ++g) {
           const float v = warp_max(mx[g]);
@@ -329,8 +329,9 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
           float v = -CUDART_INF_F;
 #pragma unroll
           for (int ww = 0; ww < kWarps; ++ww) v = fmaxf(v, s_red[ww][g]);
-          r[g] = -(v * kLog2e);
-          if (tid == g) s_ref[g] = v;                    // header value: same units as the scores
+          const float vr = v + kRefHeadroom;            // (-inf stays -inf)
+          r[g] = -(vr * kLog2e);
+          if (tid == g) s_ref[g] = vr;                   // header value: same units as the scores
         }
 #pragma unroll
         for (int j = 0; j < kW; ++j) nref2[j] = pk2(r[2 * j], GC > 1 ? r[(2 * j + 1) % GC] : 0.f);
@@ -351,7 +352,7 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
 #pragma unroll
         for (int g = 1; g < GC; ++g) xm = fmaxf(xm, x[g]);
         if (xm > kOverflowGuardLog2) s_overflow = 1;
-        if (xm > kNegligibleLog2) {
+        if (xm > kScanNegligibleLog2) {
           float e[GC];
 #pragma unroll
           for (int g = 0; g < GC; ++g) e[g] = fast_exp2(x[g]);
@@ -389,20 +390,31 @@ scan4_kernel(Plan pl, const uint8_t* __restrict__ codes, const uint16_t* __restr
       if (tid < GC) s_ref[tid] = s_max[tid];
       __threadfence();
       __syncthreads();
-      for (int i = seg_begin + tid; i < seg_end; i += kScanThreads) {
-        const uint32_t lid = min((uint32_t)__ldg(lid_row + i), (uint32_t)(n_list - 1));
-        float e[GC];
-        bool any = false;
+      // (eight tokens per thread in flight: the pass is a chain of L2 round trips otherwise)
+      constexpr int kRb = 8;
+      for (int i0 = seg_begin + tid; i0 < seg_end; i0 += kRb * kScanThreads) {
+        uint32_t lid[kRb];
+        float sv[kRb][GC];
 #pragma unroll
-        for (int g = 0; g < GC; ++g) {
-          e[g] = 0.f;
-          if (g < n_heads) {
-            const float s = __ldcg(sc_row[g] + i);
-            const float x = fmaf(s, kLog2e, -(s_ref[g] * kLog2e));     // -inf outside R
+        for (int u = 0; u < kRb; ++u) {
+          const int i = i0 + u * kScanThreads;
+          lid[u] = i < seg_end ? (uint32_t)__ldg(lid_row + i) : 0u;
+#pragma unroll
+          for (int g = 0; g < GC; ++g)
+            sv[u][g] = (g < n_heads && i < seg_end) ? __ldcg(sc_row[g] + i) : -CUDART_INF_F;
+        }
+#pragma unroll
+        for (int u = 0; u < kRb; ++u) {
+          float e[GC];
+          bool any = false;
+#pragma unroll
+          for (int g = 0; g < GC; ++g) {
+            const float x = fmaf(sv[u][g], kLog2e, -(s_ref[g] * kLog2e));     // -inf outside R
+            e[g] = 0.f;
             if (x > kNegligibleLog2) { e[g] = fast_exp2(x); any = true; }
           }
+          if (any) red_add<GC>(part_sums + (size_t)min(lid[u], (uint32_t)(n_list - 1)) * GC, e);
         }
-        if (any) red_add<GC>(part_sums + (size_t)lid * GC, e);
       }
     }
     // header: the reference the sums are relative to (same units as the scores) and the

@@ -70,6 +70,14 @@ template <int GC> __device__ __forceinline__ void red_add(float* dst, const floa
 }
 
 constexpr float kOverflowGuardLog2 = 96.0f;   // exp2 arguments above this trigger the rebuild
+// The reference of a segment's exp-sums is set this far above the maximum of the CTA's first
+// round of tiles, so that a later, larger logit (heavy-tailed keys: the maximum of 57 K tokens
+// is far above the maximum of the first 512) still lands below the overflow guard and the
+// segment is not rebuilt; terms are kept down to 2^-40 of the first round's maximum, as before.
+// exp2 arguments then run from -120 to +96, inside the fp32 range (2^-120 is a normal number).
+constexpr float kRefHeadroomLog2 = 80.0f;
+constexpr float kRefHeadroom = kRefHeadroomLog2 / kLog2e;             // in units of the scores
+constexpr float kScanNegligibleLog2 = kNegligibleLog2 - kRefHeadroomLog2;
 constexpr int kMbarSpinLimit = 1 << 22;
 
 // ---- bulk async copy global -> shared, completion on an mbarrier (TMA, no tensor map)

@@ -155,9 +155,10 @@ __device__ __forceinline__ int linear_bucket(float s, float lo, float scale) {
 }
 
 // Buckets (from the top) that hold the rank_a-th and rank_b-th largest (0-based) of the items
-// counted in `hist`; one pass over the histogram serves both ranks.
+// counted in `hist`, and the number of items in the buckets above the first of them; one pass
+// over the histogram serves both ranks.
 __device__ void find_two_buckets(const uint32_t* hist, int rank_a, int rank_b, int* s_scan,
-                                 int& bucket_a, int& bucket_b) {
+                                 int& bucket_a, int& bucket_b, int& above_a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int per = kHistBins / kSelThreads;                 // 8 bins per thread, top down
   const int hi = kHistBins - tid * per;
@@ -167,7 +168,7 @@ __device__ void find_two_buckets(const uint32_t* hist, int rank_a, int rank_b, i
   uint32_t local = 0;
 #pragma unroll
   for (int j = 0; j < 8; ++j) local += mine[j];
-  if (tid == 0) { s_scan[32] = 0; s_scan[33] = 0; }
+  if (tid == 0) { s_scan[32] = 0; s_scan[33] = 0; s_scan[34] = 0; }
   uint32_t inc = local;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -190,22 +191,23 @@ __device__ void find_two_buckets(const uint32_t* hist, int rank_a, int rank_b, i
   uint32_t run = (uint32_t)s_scan[warp] + inc - local;       // items in buckets above mine
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    if (run <= (uint32_t)rank_a && (uint32_t)rank_a < run + mine[j]) s_scan[32] = hi - 1 - j;
+    if (run <= (uint32_t)rank_a && (uint32_t)rank_a < run + mine[j]) { s_scan[32] = hi - 1 - j; s_scan[34] = (int)run; }
     if (run <= (uint32_t)rank_b && (uint32_t)rank_b < run + mine[j]) s_scan[33] = hi - 1 - j;
     run += mine[j];
   }
   __syncthreads();
   bucket_a = s_scan[32];
   bucket_b = s_scan[33];
+  above_a = s_scan[34];
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(kSelThreads)
+__global__ void __launch_bounds__(kSelThreads, 2)     // two rows per SM: 64 registers
 sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __restrict__ seq_lens,
                   int32_t* __restrict__ rowstate, int32_t* __restrict__ sel_count,
                   float* __restrict__ kth) {
   __shared__ __align__(16) uint32_t s_hist[kHistBins];
-  __shared__ int s_scan[34];
+  __shared__ int s_scan[36];
   __shared__ float s_mm[2][kSelThreads / 32];
   const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = row / pl.Hq;
@@ -272,16 +274,48 @@ sel_sample_kernel(Plan pl, const float* __restrict__ scores, const int32_t* __re
       // fall into the bottom bucket); the bracket is the outer edges of the two buckets that
       // hold the order statistics, one bucket wider on each side for the rounding of the edges.
       // Whatever the bracket is, the filter kernel checks it by counting.
-      const float scale = (float)kHistBins / (mx - mn);
+      // If both order statistics land within a few buckets of each other, the range was
+      // stretched by outliers (one score at -1e6 puts every other score into one bucket): the
+      // histogram is then repeated over the span of those buckets, with the samples above it
+      // counted as ranked higher, up to twice (4096-fold zoom each time).
+      const int rk_hi = max(r_hi, 0), rk_lo = min(r_lo, n_sample - 1);
+      float lo_r = mn, hi_r = mx;
+      uint32_t alive = 0u;                         // samples inside the current range
 #pragma unroll
-      for (int e = 0; e < kSamplePer; ++e)
-        if (s[e] == s[e]) atomicAdd(&s_hist[linear_bucket(s[e], mn, scale)], 1u);
-      __syncthreads();
-      int b_hi, b_lo;
-      find_two_buckets(s_hist, max(r_hi, 0), min(r_lo, n_sample - 1), s_scan, b_hi, b_lo);
-      const float width = (mx - mn) / (float)kHistBins;
-      if (r_hi >= 0) hi = mn + (float)(b_hi + 2) * width;
-      if (r_lo < n_sample && b_lo >= 2) lo = mn + (float)(b_lo - 1) * width;
+      for (int e = 0; e < kSamplePer; ++e) alive |= (s[e] == s[e] ? 1u : 0u) << e;
+      int above = 0;                               // samples ranked above the current range
+      for (int pass = 0;; ++pass) {
+        const float scale = (float)kHistBins / (hi_r - lo_r);
+        const float width = (hi_r - lo_r) / (float)kHistBins;
+#pragma unroll
+        for (int e = 0; e < kSamplePer; ++e)
+          if ((alive >> e) & 1u) atomicAdd(&s_hist[linear_bucket(s[e], lo_r, scale)], 1u);
+        __syncthreads();
+        int b_hi, b_lo, above_hi;
+        find_two_buckets(s_hist, rk_hi - above, rk_lo - above, s_scan, b_hi, b_lo, above_hi);
+        if (b_hi - b_lo >= 8 || pass == 2 || !(width > 0.f)) {
+          if (r_hi >= 0) hi = lo_r + (float)(b_hi + 2) * width;
+          if (r_lo < n_sample && (b_lo >= 2 || pass > 0)) lo = lo_r + (float)(b_lo - 1) * width;
+          break;
+        }
+        // zoom into buckets b_lo .. b_hi
+#pragma unroll
+        for (int e = 0; e < kSamplePer; ++e) {
+          const int bk = linear_bucket(s[e], lo_r, scale);
+          if (bk < b_lo || bk > b_hi) alive &= ~(1u << e);
+        }
+        above += above_hi;
+        const float nlo = lo_r + (float)b_lo * width, nhi = lo_r + (float)(b_hi + 1) * width;
+        if (!(nhi > nlo)) {                        // the floats between the edges ran out
+          if (r_hi >= 0) hi = lo_r + (float)(b_hi + 2) * width;
+          if (r_lo < n_sample) lo = lo_r + (float)(b_lo - 1) * width;
+          break;
+        }
+        lo_r = nlo;
+        hi_r = nhi;
+        for (int i = tid; i < kHistBins; i += kSelThreads) s_hist[i] = 0u;
+        __syncthreads();
+      }
     } else if (mx == mn) {
       hi = mx;                                     // all finite samples equal: take that value
       lo = mn;                                     // as the whole bracket

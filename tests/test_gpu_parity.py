@@ -367,6 +367,36 @@ def test_rows_that_defeat_the_sample_fall_back_to_the_exact_path():
     assert sorted(got[0, :k].tolist()) == sorted(hidden.tolist())
 
 
+def test_rows_with_outliers_at_sampled_positions_keep_the_exact_top_k():
+    """One score at -1e6 (or +1e6, or a handful of large ones) at positions the sample reads stretches
+    the range of the sample's histogram until every other score shares a bucket; the sample kernel
+    then zooms into the buckets that hold its order statistics.  The result is the exact top-k
+    either way (this checks the zoomed brackets; the speed is the benchmark's business)."""
+    cfg = small("outl", seq_lens=(65536,), n_q_heads=4, n_kv_heads=1, budget_ppm=10000,
+                kmeans_iters=1, n_list=16)
+    inp, idx = make_case(cfg, device="cuda")
+    op = DecodeOp(inp, idx)
+    op.alloc_stage_buffers()
+    N = op.params.max_seq_len
+    k = O.budget_k(N, 10000)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    sc = torch.randn((4, N), generator=g, device="cuda")
+    seen = torch.from_numpy(sampled_positions(N)).cuda()
+    sc[0, seen[5]] = -1e6
+    sc[1, seen[7]] = 1e6
+    sc[2, seen[::97]] *= 300.0                     # heavy tails on both sides
+    sc[3, seen[3]] = -3e38
+    sc[3, seen[4]] = 3e38                          # the range overflows to inf: no bracket, still exact
+    op.scores.view(1, 4, N)[0] = sc
+    op.select()
+    torch.cuda.synchronize()
+    assert op.device_status() == pqhsa.OK
+    got = op.sel_idx.view(4, -1).cpu().numpy()
+    for h in range(4):
+        want = O.select_topk(sc[h].cpu().double().numpy(), k)
+        assert sorted(got[h, :k].tolist()) == want.tolist()
+
+
 def test_invalid_arguments_launch_nothing():
     inp, idx, arrays, ref, op = get_case("c1")
     bad = pqhsa.Params.from_buffer_copy(op.params)

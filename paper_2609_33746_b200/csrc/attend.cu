@@ -25,6 +25,7 @@
 // preparation.  Nothing may be added above those waits that returns early.
 #include "attn_common.cuh"
 #include "common.cuh"
+#include "scan_common.cuh"
 
 namespace pqhsa {
 
@@ -46,7 +47,7 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
                const uint16_t* __restrict__ lids, const int32_t* __restrict__ seq_lens,
                float* __restrict__ bg_mass, float* __restrict__ bg_max,
                float* __restrict__ bg_aux, int32_t* __restrict__ bg_tcount) {
-  __shared__ float s_scale[kMaxSeg];
+  __shared__ float s_scale[kMaxSeg], s_ref2[kMaxSeg];
   const int row = blockIdx.y, c = blockIdx.x, C = gridDim.x, tid = threadIdx.x;
   const int b = row / pl.Hq, h = row % pl.Hq;
   const int kv = h / pl.G, hg = (h % pl.G) / pl.Gc;
@@ -135,6 +136,7 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
     // a segment's sums are relative to its reference: exp2(l~ log2 e - ref log2 e)
     const float ref = pr[(size_t)sg * seg_stride + g];
     s_scale[sg] = s_scale[sg] > -CUDART_INF_F ? fast_exp2(ref * kLog2e - m2) : 0.f;
+    s_ref2[sg] = __fmul_rn(ref, kLog2e);           // the scan's own product, rounded as there
   }
   __syncthreads();
   const int jl = (int)((long long)c * n_list / C), jh = (int)((long long)(c + 1) * n_list / C);
@@ -152,22 +154,24 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
     }
     if (acc != 0.f) atomicAdd(&mass[j], acc);
   }
-  // take the selected tokens out of their lists' sums
+  // Take the selected tokens out of their lists' sums.  A selected token can hold nearly all of
+  // its list's mass, and what is left after the subtraction is multiplied by the list's mean
+  // value, so the term taken out is formed exactly as the scan formed the term it put in (the
+  // exponent against the reference of the token's own segment, the same instructions) and
+  // scaled like that segment's sums: what remains is the rounding of the additions alone.
+  auto take_out = [&](int i, float s, uint32_t lid) {
+    const int sg = min(nseg - 1, max(0, split_cta_of(sp, s_u + i / kTile) - c_first));
+    const float x = fmaf(s, kLog2e, -s_ref2[sg]);
+    if (x > kScanNegligibleLog2) atomicAdd(&mass[lid], -(fast_exp2(x) * s_scale[sg]));
+    if (bg_tcount != nullptr) atomicAdd(&bg_tcount[(size_t)row * n_list + lid], 1);
+  };
 #pragma unroll
-  for (int u = 0; u < kSelPer; ++u) {
-    if (idx[u] >= 0) {
-      const float x = fmaf(sc[u], kLog2e, -m2);
-      if (x > kNegligibleLog2) atomicAdd(&mass[li[u]], -fast_exp2(x));
-      if (bg_tcount != nullptr) atomicAdd(&bg_tcount[(size_t)row * n_list + li[u]], 1);
-    }
-  }
+  for (int u = 0; u < kSelPer; ++u)
+    if (idx[u] >= 0) take_out(idx[u], sc[u], li[u]);
   for (int t = tl + kSelPer * kBgThreads + tid; t < th; t += kBgThreads) {
     const int i = sel[t];
     if ((unsigned)i >= (unsigned)n) continue;
-    const uint32_t lid = min((uint32_t)rl[i], (uint32_t)(n_list - 1));
-    const float x = fmaf(rs[i], kLog2e, -m2);
-    if (x > kNegligibleLog2) atomicAdd(&mass[lid], -fast_exp2(x));
-    if (bg_tcount != nullptr) atomicAdd(&bg_tcount[(size_t)row * n_list + lid], 1);
+    take_out(i, rs[i], min((uint32_t)rl[i], (uint32_t)(n_list - 1)));
   }
   if (c == 0 && tid == 0) bg_max[row] = m;
 }

@@ -48,6 +48,7 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
                float* __restrict__ bg_mass, float* __restrict__ bg_max,
                float* __restrict__ bg_aux, int32_t* __restrict__ bg_tcount) {
   __shared__ float s_scale[kMaxSeg], s_ref2[kMaxSeg];
+  __shared__ int s_segend[kMaxSeg];      // first tile of the row (32-token units) past segment sg
   const int row = blockIdx.y, c = blockIdx.x, C = gridDim.x, tid = threadIdx.x;
   const int b = row / pl.Hq, h = row % pl.Hq;
   const int kv = h / pl.G, hg = (h % pl.G) / pl.Gc;
@@ -137,6 +138,7 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
     const float ref = pr[(size_t)sg * seg_stride + g];
     s_scale[sg] = s_scale[sg] > -CUDART_INF_F ? fast_exp2(ref * kLog2e - m2) : 0.f;
     s_ref2[sg] = __fmul_rn(ref, kLog2e);           // the scan's own product, rounded as there
+    s_segend[sg] = sg + 1 < nseg ? (int)(split_start(sp, c_first + sg + 1) - s_u) : 0x7fffffff;
   }
   __syncthreads();
   const int jl = (int)((long long)c * n_list / C), jh = (int)((long long)(c + 1) * n_list / C);
@@ -159,8 +161,14 @@ bg_prep_kernel(Plan pl, const float* __restrict__ scores, const float* __restric
   // value, so the term taken out is formed exactly as the scan formed the term it put in (the
   // exponent against the reference of the token's own segment, the same instructions) and
   // scaled like that segment's sums: what remains is the rounding of the additions alone.
+  const float inv_seg_tiles = (float)sp.P_eff / (float)sp.T;          // segments per tile
+  const float tile_off = (float)(s_u - split_start(sp, c_first));     // tiles of segment 0 before this unit
   auto take_out = [&](int i, float s, uint32_t lid) {
-    const int sg = min(nseg - 1, max(0, split_cta_of(sp, s_u + i / kTile) - c_first));
+    // segments are equally long up to one tile: estimate, then settle against the boundaries
+    const int tile = i / kTile;
+    int sg = min(nseg - 1, max(0, (int)(((float)tile + tile_off) * inv_seg_tiles)));
+    while (sg > 0 && tile < s_segend[sg - 1]) --sg;
+    while (tile >= s_segend[sg]) ++sg;             // (the last entry is INT_MAX)
     const float x = fmaf(s, kLog2e, -s_ref2[sg]);
     if (x > kScanNegligibleLog2) atomicAdd(&mass[lid], -(fast_exp2(x) * s_scale[sg]));
     if (bg_tcount != nullptr) atomicAdd(&bg_tcount[(size_t)row * n_list + lid], 1);

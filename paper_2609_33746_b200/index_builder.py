@@ -67,11 +67,13 @@ def _kmeans(x: torch.Tensor, k: int, iters: int, gen: torch.Generator):
         c[:n] = x
     for _ in range(iters):
         ids, dist = _assign(x, c)
-        sums = torch.zeros_like(c).index_add_(0, ids, x)
-        cnt = torch.zeros(k, dtype=x.dtype, device=x.device).index_add_(
-            0, ids, torch.ones(n, dtype=x.dtype, device=x.device))
+        # sums in float64: the device adds in no fixed order, and at that precision the order
+        # no longer reaches the fp32 centres, so two builds of one workload give one index
+        sums = torch.zeros(c.shape, dtype=torch.float64, device=x.device).index_add_(0, ids, x.double())
+        cnt = torch.zeros(k, dtype=torch.float64, device=x.device).index_add_(
+            0, ids, torch.ones(n, dtype=torch.float64, device=x.device))
         nonempty = cnt > 0
-        c[nonempty] = sums[nonempty] / cnt[nonempty, None]
+        c[nonempty] = (sums[nonempty] / cnt[nonempty, None]).to(c.dtype)
         n_empty = int((~nonempty).sum())
         if n_empty and n > k:
             far = torch.topk(dist, n_empty).indices
@@ -90,13 +92,16 @@ def _batched_pq_kmeans(res: torch.Tensor, ncode: int, iters: int, gen: torch.Gen
     else:
         c = torch.zeros((M, ncode, dsub), dtype=res.dtype, device=res.device)
         c[:, :n] = x
-    ones = torch.ones((M, n), dtype=res.dtype, device=res.device)
+    ones = torch.ones((M, n), dtype=torch.float64, device=res.device)
+    x64 = x.double()
     for _ in range(iters):
         ids = _pq_encode(x, c, chunk)                     # [M, n]
-        sums = torch.zeros_like(c).scatter_add_(1, ids[..., None].expand(-1, -1, dsub), x)
-        cnt = torch.zeros((M, ncode), dtype=res.dtype, device=res.device).scatter_add_(1, ids, ones)
+        # (float64 sums, as in _kmeans: the order of the device's additions stays below fp32)
+        sums = torch.zeros(c.shape, dtype=torch.float64, device=res.device).scatter_add_(
+            1, ids[..., None].expand(-1, -1, dsub), x64)
+        cnt = torch.zeros((M, ncode), dtype=torch.float64, device=res.device).scatter_add_(1, ids, ones)
         ne = cnt > 0
-        c = torch.where(ne[..., None], sums / cnt.clamp(min=1)[..., None], c)
+        c = torch.where(ne[..., None], (sums / cnt.clamp(min=1)[..., None]).to(c.dtype), c)
     return c
 
 

@@ -84,3 +84,26 @@ def test_full_size_decode_on_sampled_rows(name, rows):
                 f"{name} output row {(b, h)}: max-abs {err.max()}"
     del op, inp, idx
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("variant", ["T", "Bx", "C", "C2", "C2b"])
+def test_full_size_mechanism_variants(variant):
+    """The ablation variants (Table 2, App. B) at 128K under the paper's own partition and index
+    setting, every row: the output against the oracle's for that variant."""
+    cfg = dataclasses.replace(config_of("c3p_b1_r1"), kmeans_iters=2)
+    inp = generate(cfg, device="cuda")
+    idx = build_index(inp)
+    op = DecodeOp(inp, idx, variant=variant)
+    out = op.decode()
+    torch.cuda.synchronize()
+    assert op.device_status() == pqhsa.OK
+    arrays = oracle_arrays_for_sequence(inp, idx, 0)
+    ref = run_oracle(inp, None, heads=list(ALL), batch_items=[0], arrays=arrays, variant=variant)
+    for h in ALL:
+        r = ref[(0, h)]
+        y = out[0, h].cpu().double().numpy()
+        err = np.abs(y - r["y"])
+        assert np.all(err <= out_tolerance(r["y"], cfg.dtype)), \
+            f"variant {variant} output row {(0, h)}: max-abs {err.max()}"
+    del op, inp, idx
+    torch.cuda.empty_cache()

@@ -175,8 +175,10 @@ typedef enum {
   PQHSA_BUF_BG_MASS = 7,        /* float   [B][H_q][n_list]  background mass M_j of Eq. 4,      */
                                 /*         relative to exp(BG_MAX); may be slightly negative    */
                                 /*         where every member of a list was selected (read as 0) */
-  PQHSA_BUF_BG_MAX = 8          /* float   [B][H_q]  max approximate logit of the row (-inf:    */
+  PQHSA_BUF_BG_MAX = 8,         /* float   [B][H_q]  max approximate logit of the row (-inf:    */
                                 /*         no background)                                       */
+  PQHSA_BUF_OUT_F32 = 9         /* float   [B][H_q][128]  what pqhsa_decode computed before it   */
+                                /*         rounded it to the output dtype (fused call only)     */
 } pqhsa_buffer;
 
 /* Query heads of a group are processed Gc at a time (Gc = G for G <= 2, else 4); a group

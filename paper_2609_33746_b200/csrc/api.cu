@@ -162,6 +162,7 @@ static size_t buffer_elems(const Plan& pl, int which) {
     case PQHSA_BUF_KTH: return (size_t)pl.rows;
     case PQHSA_BUF_BG_MASS: return (size_t)pl.rows * pl.n_list;
     case PQHSA_BUF_BG_MAX: return (size_t)pl.rows;
+    case PQHSA_BUF_OUT_F32: return (size_t)pl.rows * kHeadDim;
     default: return 0;
   }
 }
@@ -197,6 +198,7 @@ void make_layout(const Plan& pl, WsLayout* L) {
   L->sel_idx = take(buffer_elems(pl, PQHSA_BUF_SEL_IDX) * 4);
   L->sel_count = take(buffer_elems(pl, PQHSA_BUF_SEL_COUNT) * 4);
   L->kth = take(buffer_elems(pl, PQHSA_BUF_KTH) * 4);
+  L->out_f32 = take(buffer_elems(pl, PQHSA_BUF_OUT_F32) * 4);
   L->total = o;
 }
 
@@ -286,6 +288,7 @@ size_t pqhsa_decode_buffer_offset(const pqhsa_params* params, int which) {
     case PQHSA_BUF_KTH: return L.kth;
     case PQHSA_BUF_BG_MASS: return L.bg_mass;
     case PQHSA_BUF_BG_MAX: return L.bg_max;
+    case PQHSA_BUF_OUT_F32: return L.out_f32;
     default: return (size_t)-1;
   }
 }
@@ -435,7 +438,7 @@ static int decode_impl(const pqhsa_params* params, const void* q, const pqhsa_in
   if (e == cudaSuccess) e = mark(3);
   if (e == cudaSuccess)
     e = launch_attend(pl, L, w, q, *kv, *index, scores, partials, sel_idx, sel_count, seq_lens,
-                      out, nullptr, nullptr, st);
+                      out, nullptr, reinterpret_cast<float*>(w + L.out_f32), st);
   if (e == cudaSuccess) e = mark(4);
   return cuda_status(e);
 }

@@ -75,7 +75,7 @@ struct WsLayout {
   size_t norm_seg;                   // float  [units][n_part]: largest key norm per scan segment (fp16 tables)
   size_t stage_end;                  // end of what a single stage call needs
   // intermediates of the fused entry point
-  size_t lut, coarse, scores, list_partials, sel_idx, sel_count, kth;
+  size_t lut, coarse, scores, list_partials, sel_idx, sel_count, kth, out_f32;
   size_t total;
 };
 

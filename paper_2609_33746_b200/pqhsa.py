@@ -21,7 +21,7 @@ LIB_PATH = os.environ.get("PQHSA_LIBRARY") or os.path.join(_HERE, "libpqhsa.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_CHECK = 0, -1, -2, -3, -4, -5
 F16, BF16 = 0, 1
 (BUF_LUT, BUF_COARSE, BUF_SCORES, BUF_LIST_PARTIALS, BUF_SEL_IDX, BUF_SEL_COUNT, BUF_KTH,
- BUF_BG_MASS, BUF_BG_MAX) = range(9)
+ BUF_BG_MASS, BUF_BG_MAX, BUF_OUT_F32) = range(10)
 VARIANTS = {"B": 0, "T": 1, "Bx": 2, "C": 3, "C2": 4, "C2b": 5}      # pqhsa_variant
 
 EXPORTS = [

@@ -14,7 +14,7 @@ from paper_2609_33746_b200.runner import DecodeOp
 from paper_2609_33746_b200.workload import generate, named_config
 
 from helpers import oracle_arrays_for_sequence, run_oracle, selection_matches
-from test_gpu_parity import LOGIT_RTOL, out_tolerance
+from test_gpu_parity import LOGIT_RTOL, OUT_ATOL, half_ulp, out_tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -58,6 +58,7 @@ def test_full_size_decode_on_sampled_rows(name, rows):
     scores = op.decode_buffer(pqhsa.BUF_SCORES).view(cfg.batch, cfg.n_q_heads, N_max)
     sel = op.decode_buffer(pqhsa.BUF_SEL_IDX, torch.int32).view(cfg.batch, cfg.n_q_heads, k_max)
     cnt = op.decode_buffer(pqhsa.BUF_SEL_COUNT, torch.int32).view(cfg.batch, cfg.n_q_heads)
+    out32 = op.decode_buffer(pqhsa.BUF_OUT_F32).view(cfg.batch, cfg.n_q_heads, -1)   # before the rounding
     by_seq = {}
     for b, h in rows:
         by_seq.setdefault(b, []).append(h)
@@ -78,10 +79,12 @@ def test_full_size_decode_on_sampled_rows(name, rows):
                 assert (c + r0 + (n - r1)) % cfg.exact_set_multiple == 0
             ok, why = selection_matches(sel[b, h, :c].cpu().numpy(), r)
             assert ok, f"{name} selection row {(b, h)}: {why}"
+            y32 = out32[b, h].cpu().double().numpy()
+            assert np.abs(y32 - r["y"]).max() <= OUT_ATOL, \
+                f"{name} output row {(b, h)} before rounding: max-abs {np.abs(y32 - r['y']).max()}"
             y = out[b, h].cpu().double().numpy()
-            err = np.abs(y - r["y"])
-            assert np.all(err <= out_tolerance(r["y"], cfg.dtype)), \
-                f"{name} output row {(b, h)}: max-abs {err.max()}"
+            assert np.all(np.abs(y - y32) <= half_ulp(y32, cfg.dtype) * 1.0001), \
+                f"{name} stored output row {(b, h)} is not the computed one rounded"
     del op, inp, idx
     torch.cuda.empty_cache()
 
@@ -99,11 +102,13 @@ def test_full_size_mechanism_variants(variant):
     assert op.device_status() == pqhsa.OK
     arrays = oracle_arrays_for_sequence(inp, idx, 0)
     ref = run_oracle(inp, None, heads=list(ALL), batch_items=[0], arrays=arrays, variant=variant)
+    out32 = op.decode_buffer(pqhsa.BUF_OUT_F32).view(cfg.batch, cfg.n_q_heads, -1)
     for h in ALL:
         r = ref[(0, h)]
+        y32 = out32[0, h].cpu().double().numpy()
+        assert np.abs(y32 - r["y"]).max() <= OUT_ATOL, \
+            f"variant {variant} output row {(0, h)} before rounding: max-abs {np.abs(y32 - r['y']).max()}"
         y = out[0, h].cpu().double().numpy()
-        err = np.abs(y - r["y"])
-        assert np.all(err <= out_tolerance(r["y"], cfg.dtype)), \
-            f"variant {variant} output row {(0, h)}: max-abs {err.max()}"
+        assert np.all(np.abs(y - r["y"]) <= out_tolerance(r["y"], cfg.dtype))
     del op, inp, idx
     torch.cuda.empty_cache()
